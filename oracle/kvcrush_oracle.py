@@ -1,0 +1,343 @@
+"""TEST INFRASTRUCTURE - float64 CPU oracle for the KVCrush compression pass.
+
+Not part of the product.  Only the tests, the smoke check and the CPU-baseline
+leg of the benchmark may import this module; it shares no code with the CUDA
+library and never calls it.
+
+Every function restates one step of the paper in plain numpy (the score step
+can also run through the plain C routine in ``score_oracle.c`` which is the
+same definition, row by row, for sizes numpy would be too slow for).  KVCrush is
+a heuristic, so the oracle is the algorithm taken step by step:
+
+  O1  A_h = softmax(Q_h K_h^T / sqrt(d_k))                     Algorithm 1
+  O2  c_h(t) = sum_j A_h(j, t)   (w_h(t) = c_h(t) / S)          Algorithm 1, Sec. 3.1
+  O3  theta_h, b_t[h] = [w_h(t) >= theta_h], packed             Algorithm 1, Sec. 3.1
+  O4  B_important tokens by cumulative attention (H2O)         Sec. 3, Sec. 4.1.1
+  O5  anchor a, d_t = Hamming(b_t, a)                           Algorithm 2, Sec. 3.2
+  O6  B_representative buckets by d_t                           Algorithm 2, Sec. 3.2
+  O7  representative = member closest to the bucket centroid   Algorithm 2, Sec. 3.2
+  O8  kept = important U representatives                        Sec. 3.2
+  O9  reduced cache = kept rows of K and V                      Sec. 3.2
+
+Readings taken where the paper is silent or garbled (each one is a single
+function or parameter here):
+
+* column sums, not the row sums the printed index order would give (``scores``);
+* theta_h is the k-th largest score of head h, k = total budget by default
+  (``thresholds``) - PARITY UNPINNED by the paper: it only says the threshold
+  keeps a target fraction of tokens per head;
+* the importance of a token is the sum of its per-head scores, accumulated in
+  float64 head by head in ascending order, KV group by KV group
+  (``importance``); ties go to the lower token index;
+* the tokens that are grouped are those NOT kept as important
+  (``select``) - PARITY UNPINNED: Algorithm 2 lists all S tokens as input while
+  Sec. 3 calls the representatives proxies of the evicted tokens;
+* anchors: alternate = bit h is h mod 2; mean = per-bit majority over the
+  grouped tokens, ties to 1; explicit bits cover "random" (``anchor_bits``)
+  - the first bit of the alternating pattern and the population of the mean are
+  PARITY UNPINNED;
+* buckets are equal-frequency: sort the grouped tokens by (d_t, t) and cut the
+  order into B_representative contiguous runs (``bucket_bounds``) - PARITY
+  UNPINNED: the paper says "based on d_t" only, but d_t takes at most H+1
+  values so only this reading yields exactly one representative per bucket and
+  exactly B kept tokens;
+* the centroid is the per-bit mean and "closest" is L1 (equivalently squared
+  L2) distance, evaluated as an exact integer cost (``representative``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_C_SRC = os.path.join(_HERE, "score_oracle.c")
+_C_LIB = os.path.join(_HERE, "libscore_oracle.so")
+
+ANCHOR_ALTERNATE = 0
+ANCHOR_MEAN = 1
+ANCHOR_EXPLICIT = 2
+
+
+# ---------------------------------------------------------------------------
+# O1-O2  scores
+# ---------------------------------------------------------------------------
+
+def build_c(force: bool = False) -> str:
+    """Compile ``score_oracle.c`` (gcc, OpenMP, no fast-math) next to its source."""
+    if force or not os.path.exists(_C_LIB) or os.path.getmtime(_C_LIB) < os.path.getmtime(_C_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", _C_LIB, _C_SRC, "-lm"])
+    return _C_LIB
+
+
+_lib = None
+
+
+def _c_lib():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build_c())
+        lib.kvcrush_oracle_scores.restype = ctypes.c_int
+        lib.kvcrush_oracle_scores.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            ctypes.c_int, ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p]
+        lib.kvcrush_oracle_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def n_threads() -> int:
+    return int(_c_lib().kvcrush_oracle_threads())
+
+
+def scores(q: np.ndarray, k: np.ndarray, causal: bool = True, scale: Optional[float] = None,
+           normalize: bool = False) -> Tuple[np.ndarray, np.ndarray]:
+    """Column sums of the softmax attention matrix, one sequence (Algorithm 1).
+
+    q [L, Hq, D], k [L, Hkv, D] float64.  Returns (c [Hq, L], lse [Hq, L]) float64;
+    with ``normalize`` the first is w = c / L.  Runs the C routine (row by row).
+    """
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k = np.ascontiguousarray(k, dtype=np.float64)
+    L, Hq, D = q.shape
+    Hkv = k.shape[1]
+    assert k.shape == (L, Hkv, D) and Hq % Hkv == 0
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    c = np.zeros((Hq, L), dtype=np.float64)
+    lse = np.zeros((Hq, L), dtype=np.float64)
+    rc = _c_lib().kvcrush_oracle_scores(q.ctypes.data, k.ctypes.data, L, Hq, Hkv, D, int(bool(causal)),
+                                        float(scale), c.ctypes.data, lse.ctypes.data)
+    if rc != 0:
+        raise RuntimeError("kvcrush_oracle_scores failed")
+    if normalize and L > 0:
+        c = c / L
+    return c, lse
+
+
+def attention_matrix(q: np.ndarray, k: np.ndarray, causal: bool = True,
+                     scale: Optional[float] = None) -> np.ndarray:
+    """Brute force: the explicit [Hq, L, L] softmax matrices A_h(j, t) (small L only)."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    L, Hq, D = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    A = np.zeros((Hq, L, L), dtype=np.float64)
+    for h in range(Hq):
+        S = scale * (q[:, h, :] @ k[:, h // G, :].T)
+        if causal:
+            S = np.where(np.tril(np.ones((L, L), dtype=bool)), S, -np.inf)
+        S = S - S.max(axis=1, keepdims=True)
+        E = np.exp(S)
+        A[h] = E / E.sum(axis=1, keepdims=True)
+    return A
+
+
+def scores_bruteforce(q, k, causal=True, scale=None, normalize=False) -> np.ndarray:
+    """c_h(t) = sum_j A_h(j, t) from the explicit matrices (small L only)."""
+    A = attention_matrix(q, k, causal, scale)
+    c = A.sum(axis=1)
+    return c / q.shape[0] if normalize else c
+
+
+def to_scores32(c: np.ndarray) -> np.ndarray:
+    """The float32 array on which the signature and selection steps are defined."""
+    return np.asarray(c, dtype=np.float64).astype(np.float32)
+
+
+# ---------------------------------------------------------------------------
+# O3  thresholds and signatures
+# ---------------------------------------------------------------------------
+
+def thresholds(scores32: np.ndarray, keep: int) -> np.ndarray:
+    """theta_h = the ``keep``-th largest value of head h (Sec. 3.1: the threshold keeps
+    a target fraction of the tokens of each head).  keep >= L -> -inf (all ones);
+    keep <= 0 -> +inf (all zeros)."""
+    Hq, L = scores32.shape
+    if keep <= 0:
+        return np.full(Hq, np.inf, dtype=np.float32)
+    if keep >= L:
+        return np.full(Hq, -np.inf, dtype=np.float32)
+    srt = np.sort(scores32, axis=1)[:, ::-1]
+    return np.ascontiguousarray(srt[:, keep - 1]).astype(np.float32)
+
+
+def signatures(scores32: np.ndarray, theta: np.ndarray) -> np.ndarray:
+    """b_t[h] = 1 iff score_h(t) >= theta_h (Algorithm 1), packed: head h is bit
+    h mod 32 of word h div 32.  Returns uint32 [L, W]."""
+    Hq, L = scores32.shape
+    W = (Hq + 31) // 32
+    sig = np.zeros((L, W), dtype=np.uint32)
+    for h in range(Hq):
+        bit = (scores32[h] >= np.float32(theta[h])).astype(np.uint32)
+        sig[:, h // 32] |= bit << np.uint32(h % 32)
+    return sig
+
+
+# ---------------------------------------------------------------------------
+# O4  importance (H2O)
+# ---------------------------------------------------------------------------
+
+def importance(scores32: np.ndarray, n_kv_heads: int) -> np.ndarray:
+    """I(t): sum of the per-head scores, float64, heads added one at a time in
+    ascending order inside each KV group, then the group sums in ascending order."""
+    Hq, L = scores32.shape
+    G = Hq // n_kv_heads
+    total = np.zeros(L, dtype=np.float64)
+    for g in range(n_kv_heads):
+        group = np.zeros(L, dtype=np.float64)
+        for h in range(g * G, (g + 1) * G):
+            group = group + scores32[h].astype(np.float64)
+        total = total + group
+    return total
+
+
+def top_important(I: np.ndarray, b_imp: int) -> np.ndarray:
+    """Token ids of the b_imp largest I, ties to the lower index; returned ascending."""
+    L = I.shape[0]
+    order = np.lexsort((np.arange(L), -I))       # primary -I ascending, secondary index ascending
+    return np.sort(order[: max(0, min(b_imp, L))]).astype(np.int64)
+
+
+# ---------------------------------------------------------------------------
+# O5  anchor and Hamming distance
+# ---------------------------------------------------------------------------
+
+def _head_mask(n_q_heads: int) -> np.ndarray:
+    W = (n_q_heads + 31) // 32
+    m = np.full(W, 0xFFFFFFFF, dtype=np.uint32)
+    tail = n_q_heads - 32 * (W - 1)
+    if tail < 32:
+        m[-1] = np.uint32((1 << tail) - 1)
+    return m
+
+
+def unpack_bits(sig: np.ndarray, n_q_heads: int) -> np.ndarray:
+    """[N, W] uint32 -> [N, Hq] array of 0/1."""
+    N = sig.shape[0]
+    out = np.zeros((N, n_q_heads), dtype=np.int64)
+    for h in range(n_q_heads):
+        out[:, h] = (sig[:, h // 32] >> np.uint32(h % 32)) & np.uint32(1)
+    return out
+
+
+def pack_bits(bits: np.ndarray) -> np.ndarray:
+    n_q_heads = bits.shape[-1]
+    W = (n_q_heads + 31) // 32
+    out = np.zeros(W, dtype=np.uint32)
+    for h in range(n_q_heads):
+        if bits[h]:
+            out[h // 32] |= np.uint32(1) << np.uint32(h % 32)
+    return out
+
+
+def anchor_bits(mode: int, n_q_heads: int, cand_sigs: Optional[np.ndarray] = None,
+                explicit: Optional[np.ndarray] = None) -> np.ndarray:
+    """Anchor a in {0,1}^H (Algorithm 2): alternating 0-1 (head 0 -> 0), per-bit mean of
+    the grouped vectors rounded to a bit (ties -> 1), or caller-supplied bits."""
+    if mode == ANCHOR_ALTERNATE:
+        return pack_bits(np.arange(n_q_heads) % 2)
+    if mode == ANCHOR_MEAN:
+        bits = unpack_bits(cand_sigs, n_q_heads)
+        N = bits.shape[0]
+        return pack_bits((2 * bits.sum(axis=0) >= N).astype(np.int64))
+    if mode == ANCHOR_EXPLICIT:
+        return (np.asarray(explicit, dtype=np.uint32) & _head_mask(n_q_heads)).astype(np.uint32)
+    raise ValueError(mode)
+
+
+def hamming(sig: np.ndarray, anchor: np.ndarray, n_q_heads: int) -> np.ndarray:
+    """d_t = number of heads on which b_t and a differ."""
+    diff = unpack_bits(sig, n_q_heads) != unpack_bits(anchor[None, :], n_q_heads)
+    return diff.sum(axis=1).astype(np.int64)
+
+
+# ---------------------------------------------------------------------------
+# O6-O7  buckets and representatives
+# ---------------------------------------------------------------------------
+
+def bucket_bounds(N: int, R: int) -> np.ndarray:
+    """Equal-frequency cut of N sorted positions into R runs: run i is
+    [floor(i*N/R), floor((i+1)*N/R))."""
+    return np.asarray([(i * N) // R for i in range(R + 1)], dtype=np.int64)
+
+
+def representative(member_tokens: np.ndarray, member_sigs: np.ndarray, n_q_heads: int) -> int:
+    """The member whose vector is closest to the bucket centroid (Algorithm 2).
+
+    Centroid c[h] = n_h / m.  For a 0/1 vector b, |b - c|_1 = sum_h c[h] + sum_{h: b[h]=1} (1 - 2 c[h]),
+    so ranking by distance is ranking by the integer  sum_{h: b[h]=1} (m - 2 n_h).
+    Ties go to the lower token index."""
+    bits = unpack_bits(member_sigs, n_q_heads)
+    m = bits.shape[0]
+    n_h = bits.sum(axis=0)
+    cost = (bits * (m - 2 * n_h)[None, :]).sum(axis=1)
+    best = np.lexsort((member_tokens, cost))[0]
+    return int(member_tokens[best])
+
+
+# ---------------------------------------------------------------------------
+# O4-O8  selection of the kept set of one sequence
+# ---------------------------------------------------------------------------
+
+def select(scores32: np.ndarray, sig: np.ndarray, b_imp: int, b_rep: int, n_kv_heads: int,
+           anchor_mode: int = ANCHOR_ALTERNATE, explicit_anchor: Optional[np.ndarray] = None):
+    """Kept token ids (ascending) and their kind (0 important, 1 representative).
+
+    A budget b_imp + b_rep >= L keeps every token (kind 0)."""
+    Hq, L = scores32.shape
+    if b_imp + b_rep >= L:
+        return np.arange(L, dtype=np.int64), np.zeros(L, dtype=np.uint8)
+    I = importance(scores32, n_kv_heads)
+    imp = top_important(I, b_imp)
+    is_imp = np.zeros(L, dtype=bool)
+    is_imp[imp] = True
+    reps = np.zeros(0, dtype=np.int64)
+    if b_rep > 0:
+        cand = np.nonzero(~is_imp)[0]
+        N = cand.shape[0]
+        a = anchor_bits(anchor_mode, Hq, sig[cand], explicit_anchor)
+        d = hamming(sig[cand], a, Hq)
+        order = np.lexsort((cand, d))                 # by d_t, then token index
+        srt = cand[order]
+        bounds = bucket_bounds(N, b_rep)
+        reps = np.asarray([representative(srt[bounds[i]:bounds[i + 1]], sig[srt[bounds[i]:bounds[i + 1]]], Hq)
+                           for i in range(b_rep)], dtype=np.int64)
+    kept = np.sort(np.concatenate([imp, reps]))
+    kind = np.zeros(kept.shape[0], dtype=np.uint8)
+    kind[np.isin(kept, reps)] = 1
+    return kept, kind
+
+
+def compact(cache: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    """Reduced cache: rows idx of a token-major cache [L, ...] (byte copy)."""
+    return np.ascontiguousarray(cache[np.asarray(idx, dtype=np.int64)])
+
+
+def compress_sequence(q, k, b_imp, b_rep, sig_keep=None, causal=True, scale=None,
+                      anchor_mode=ANCHOR_ALTERNATE, explicit_anchor=None):
+    """The whole pass for one sequence of one layer. q [L,Hq,D], k [L,Hkv,D] float64."""
+    c, lse = scores(q, k, causal, scale)
+    s32 = to_scores32(c)
+    keep = (b_imp + b_rep) if sig_keep is None else sig_keep
+    theta = thresholds(s32, keep)
+    sig = signatures(s32, theta)
+    idx, kind = select(s32, sig, b_imp, b_rep, k.shape[1], anchor_mode, explicit_anchor)
+    return dict(colsum=c, lse=lse, scores32=s32, theta=theta, sig=sig, idx=idx, kind=kind)
+
+
+# ---------------------------------------------------------------------------
+# Eq. 1
+# ---------------------------------------------------------------------------
+
+def kv_memory_bytes(batch: int, n_layers: int, n_heads: int, seq_len: int, head_dim: int,
+                    precision_bytes: int) -> int:
+    """Eq. 1: 2 * B * N_L * N_H * L_seq * D * precision."""
+    return 2 * batch * n_layers * n_heads * seq_len * head_dim * precision_bytes
