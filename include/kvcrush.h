@@ -1,0 +1,202 @@
+/*
+ * kvcrush.h - C ABI of the B200 (sm_100a) KVCrush KV-cache compression pass.
+ *
+ * One pass over the prompt of every (layer, sequence) runs four stages:
+ *
+ *   kvcrush_score      per-token, per-head attention importance: column sums of
+ *                      the softmax attention matrix          (Algorithm 1, Sec. 3.1)
+ *   kvcrush_signature  per-head thresholds and the packed binary head-behaviour
+ *                      signature of every token              (Algorithm 1, Sec. 3.1)
+ *   kvcrush_select     B_important tokens by cumulative attention (H2O) plus one
+ *                      representative per Hamming bucket of the remaining tokens
+ *                                                            (Algorithm 2, Sec. 3, Sec. 3.2)
+ *   kvcrush_compact    gather of the kept K/V rows into the reduced cache (Sec. 3.2)
+ *
+ * Conventions for every entry point unless stated otherwise
+ *   - Pointers named *_dev (and every tensor / output pointer) are DEVICE pointers
+ *     owned by the caller; pointers named *_host are host pointers read during the
+ *     call only.  The library allocates and frees no memory and keeps no state
+ *     between calls; scratch memory is the caller's `workspace` (device, 256-byte
+ *     aligned, size from kvcrush_workspace_size).
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and the call returns without synchronising.  Inputs are never written.
+ *   - Return value: KVCRUSH_OK, or a negative KVCRUSH_ERR_* code, in which case
+ *     nothing was enqueued.  Problems found on the device (a bounded wait that ran
+ *     out) are reported through `status_dev` (int32[4], zeroed by the caller before
+ *     the first call): status[0] = 0 when fine, else a KVCRUSH_DEV_* code,
+ *     status[1] = kernel id, status[2..3] = detail.  A kernel that reports an
+ *     error leaves its outputs unspecified.
+ *   - Token-major tensors: element (layer l, token t, head h, channel d) lives at
+ *     ptr + l*stride_layer + t*stride_token + h*stride_head + d (strides in
+ *     elements, channel stride 1).  Tokens of all sequences are packed along the
+ *     token axis: sequence s owns tokens [cu_seqlens[s], cu_seqlens[s+1]).
+ *   - Per-head score arrays are [n_layers][n_q_heads][total_tokens] float32;
+ *     signatures are [n_layers][total_tokens][W] uint32, W = ceil(n_q_heads/32),
+ *     head h in bit (h mod 32) of word (h div 32), unused bits zero.
+ */
+#ifndef KVCRUSH_H_
+#define KVCRUSH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* return codes */
+#define KVCRUSH_OK                 0
+#define KVCRUSH_ERR_INVALID_ARG   (-1)   /* NULL pointer, negative size, inconsistent shapes */
+#define KVCRUSH_ERR_UNSUPPORTED   (-2)   /* shape or type outside what the kernels handle   */
+#define KVCRUSH_ERR_MISALIGNED    (-3)   /* pointer or stride breaks an alignment rule       */
+#define KVCRUSH_ERR_WORKSPACE     (-4)   /* workspace NULL or too small                      */
+#define KVCRUSH_ERR_CUDA          (-5)   /* a CUDA runtime / driver call failed              */
+
+/* status_dev[0] values */
+#define KVCRUSH_DEV_OK             0
+#define KVCRUSH_DEV_TIMEOUT        1     /* a bounded wait on a barrier ran out */
+
+/* element types */
+#define KVCRUSH_BF16  0
+#define KVCRUSH_FP16  1
+#define KVCRUSH_FP32  2
+
+/* stages, for kvcrush_workspace_size */
+#define KVCRUSH_STAGE_SCORE      0
+#define KVCRUSH_STAGE_SIGNATURE  1
+#define KVCRUSH_STAGE_SELECT     2
+#define KVCRUSH_STAGE_COMPACT    3
+
+/* anchor strategies of Algorithm 2 */
+#define KVCRUSH_ANCHOR_ALTERNATE 0   /* bit h = h mod 2 (head 0 -> 0)                         */
+#define KVCRUSH_ANCHOR_MEAN      1   /* per-bit majority of the grouped tokens, ties -> 1     */
+#define KVCRUSH_ANCHOR_EXPLICIT  2   /* caller's bits (a seeded random anchor is drawn on the host) */
+
+/* score kernels */
+#define KVCRUSH_SCORE_AUTO       0   /* tensor-core kernels when the shape allows, else SIMT  */
+#define KVCRUSH_SCORE_SIMT       1   /* fp32 CUDA-core kernels (any supported shape and type) */
+#define KVCRUSH_SCORE_TENSOR     2   /* tcgen05 kernels, error if the shape is not supported  */
+
+/* Shape of one compression problem; shared by all four stages. */
+typedef struct kvcrush_problem {
+  int32_t n_layers;               /* >= 1 */
+  int32_t n_seqs;                 /* sequences in the packed batch, >= 1 */
+  int32_t n_q_heads;              /* 1..128 */
+  int32_t n_kv_heads;             /* divides n_q_heads; query head h reads KV head h / (n_q_heads/n_kv_heads) */
+  int32_t head_dim;               /* D */
+  int32_t total_tokens;           /* T = cu_seqlens[n_seqs] */
+  int32_t max_seqlen;             /* longest sequence */
+  int32_t causal;                 /* 1: query j attends keys t <= j of its own sequence; 0: all keys of the sequence */
+  float   softmax_scale;          /* 0 => 1/sqrt(head_dim) (Algorithm 1) */
+  int32_t reserved;               /* set to 0 */
+  const int32_t* cu_seqlens_host; /* [n_seqs+1] ascending from 0; HOST copy (grid sizing) */
+  const int32_t* cu_seqlens_dev;  /* the same array in device memory */
+} kvcrush_problem_t;
+
+/* A token-major tensor [n_layers][total_tokens][heads][head_dim]. */
+typedef struct kvcrush_tensor {
+  const void* ptr_dev;            /* 16-byte aligned */
+  int32_t dtype;                  /* KVCRUSH_BF16 | KVCRUSH_FP16 | KVCRUSH_FP32 */
+  int32_t reserved;               /* set to 0 */
+  int64_t stride_layer;           /* in elements; every stride * element size must be a multiple of 16 bytes */
+  int64_t stride_token;
+  int64_t stride_head;
+} kvcrush_tensor_t;
+
+/* Bytes of device workspace `stage` needs for this problem (0 is a valid answer). */
+int kvcrush_workspace_size(const kvcrush_problem_t* problem, int stage, size_t* bytes);
+
+/*
+ * Stage 1 - attention-importance scores (Algorithm 1, first two steps).
+ *   A_h = softmax(Q_h K_h^T * softmax_scale) per sequence (causal if problem->causal),
+ *   scores[l][h][t] = sum over the queries j of t's sequence of A_h(j, t)
+ * i.e. the attention key t receives.  (Algorithm 1 prints the sum with A_h's indices
+ * in the other order, which is identically 1; the column sum is what is computed.)
+ * With normalize != 0 the result is divided by the sequence length (the paper's 1/S).
+ * The S x S matrix is never stored: a first sweep computes the log-sum-exp of every
+ * query row, a second sweep recomputes the logits and accumulates exp(s - lse).
+ *   Q, K        token-major tensors with n_q_heads / n_kv_heads heads, same dtype
+ *               (BF16 or FP32).  Tensor-core kernels: BF16, head_dim 64 or 128.
+ *   lse_in_dev  optional [n_layers][n_q_heads][T] float32 natural-log row
+ *               log-sum-exp of the scaled logits (as a prefill attention kernel
+ *               returns it); when given the first sweep is skipped.
+ *   scores_dev  out [n_layers][n_q_heads][T] float32
+ *   lse_out_dev optional out, same shape: the row log-sum-exp (natural log);
+ *               not written when lse_in_dev is given
+ *   impl        KVCRUSH_SCORE_*
+ *   workspace   kvcrush_workspace_size(.., KVCRUSH_STAGE_SCORE, ..) bytes
+ */
+int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, const kvcrush_tensor_t* K,
+                  const float* lse_in_dev, float* scores_dev, float* lse_out_dev, int normalize, int impl,
+                  void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * Stage 2 - per-head thresholds and packed signatures (Algorithm 1, Sec. 3.1).
+ *   theta[l][s][h] = the keep-th largest value of scores[l][h][tokens of s]
+ *                    (keep >= length: -inf, all ones; keep <= 0: +inf, all zeros)
+ *   bit h of sigs[l][t] = scores[l][h][t] >= theta[l][seq(t)][h]
+ *   sig_keep_dev   [n_layers][n_seqs] int32 rank per (layer, sequence); ignored when
+ *                  theta_in_dev is given
+ *   theta_in_dev   optional [n_layers][n_seqs][n_q_heads] float32 explicit thresholds
+ *                  (the input form of Algorithm 1)
+ *   sigs_dev       out [n_layers][T][W] uint32
+ *   theta_out_dev  optional out [n_layers][n_seqs][n_q_heads] float32
+ *   workspace      holds the thresholds when theta_out_dev is NULL
+ */
+int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev, const int32_t* sig_keep_dev,
+                      const float* theta_in_dev, uint32_t* sigs_dev, float* theta_out_dev,
+                      void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * Stage 3 - the kept set of every (layer, sequence) (Sec. 3, Algorithm 2, Sec. 3.2).
+ *   I(t)  = sum of the per-head scores of t: float64, heads added in ascending order
+ *           inside each KV group, then the group sums in ascending order
+ *   Imp   = the budget_imp tokens of largest I (ties: lower token index)       [H2O]
+ *   C     = the other tokens, N = |C|; anchor a; d_t = popcount(sig_t xor a)
+ *   sort C by (d_t, t); bucket i = sorted positions [floor(i*N/R), floor((i+1)*N/R)),
+ *           R = budget_rep
+ *   rep_i = member of bucket i closest to the bucket's per-bit mean (L1; ties: lower t)
+ *   kept  = Imp U {rep_i}, ascending token index.  budget_imp + budget_rep >= length
+ *           keeps every token.
+ *   budget_imp_dev, budget_rep_dev  [n_layers][n_seqs] int32, >= 0
+ *   anchor_mode        KVCRUSH_ANCHOR_*
+ *   anchor_bits_dev    [W] uint32 (anchor_per_segment == 0) or [n_layers][n_seqs][W];
+ *                      read only for KVCRUSH_ANCHOR_EXPLICIT; bits above n_q_heads ignored
+ *   cu_kept_dev        [n_layers*n_seqs + 1] int32: where each segment's kept list starts
+ *                      in idx_dev, segment = layer*n_seqs + seq; the caller sets it to the
+ *                      prefix sums of min(budget_imp + budget_rep, length)
+ *   idx_dev            out [cu_kept[last]] int32 token index inside its sequence
+ *   kind_dev           optional out, same length, uint8: 0 important, 1 representative
+ * Sequences longer than 262144 tokens are not supported.
+ */
+int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
+                   const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                   const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev,
+                   void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * Stage 4 - reduced cache (Sec. 3.2: the kept tokens form the final cache).
+ *   out[l][cu_kept[l*n_seqs+s] - cu_kept[l*n_seqs] + i][h][:] =
+ *        in[l][cu_seqlens[s] + idx[cu_kept[l*n_seqs+s] + i]][h][:]        for K and for V
+ *   K, V           token-major caches with n_kv_heads heads (any element type; bytes are copied)
+ *   total_kept     cu_kept[n_layers*n_seqs] (host value, for grid sizing)
+ *   K_out, V_out   token-major outputs; ptr_dev is written; same dtype as the inputs;
+ *                  head_dim * element size must be a multiple of 16 bytes
+ * V (and V_out) may be NULL to gather one tensor only.
+ */
+int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K, const kvcrush_tensor_t* V,
+                    const int32_t* cu_kept_dev, const int32_t* idx_dev, int64_t total_kept,
+                    const kvcrush_tensor_t* K_out, const kvcrush_tensor_t* V_out,
+                    int32_t* status_dev, void* stream);
+
+/* Text for a return code. */
+const char* kvcrush_strerror(int code);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int kvcrush_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVCRUSH_H_ */

@@ -1,0 +1,183 @@
+// extern "C" entry points of the kvcrush library: argument validation and stage dispatch.
+// Every check that can fail happens before the first launch, so an error return means nothing ran.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace {
+
+using namespace kvc;
+
+constexpr size_t kAlign = 256;
+inline size_t round_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+int make_shape(const kvcrush_problem_t* p, Shape* s) {
+  if (!p) return KVCRUSH_ERR_INVALID_ARG;
+  if (p->n_layers < 1 || p->n_seqs < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->head_dim < 1 ||
+      p->total_tokens < 0 || p->max_seqlen < 0)
+    return KVCRUSH_ERR_INVALID_ARG;
+  if (p->n_q_heads % p->n_kv_heads != 0) return KVCRUSH_ERR_INVALID_ARG;
+  if (p->n_q_heads > 128) return KVCRUSH_ERR_UNSUPPORTED;
+  if (!p->cu_seqlens_host || !p->cu_seqlens_dev) return KVCRUSH_ERR_INVALID_ARG;
+  const int32_t* cu = p->cu_seqlens_host;
+  if (cu[0] != 0 || cu[p->n_seqs] != p->total_tokens) return KVCRUSH_ERR_INVALID_ARG;
+  for (int i = 0; i < p->n_seqs; ++i) {
+    const int len = cu[i + 1] - cu[i];
+    if (len < 0 || len > p->max_seqlen) return KVCRUSH_ERR_INVALID_ARG;
+  }
+  if ((long long)p->n_layers * p->n_q_heads * (long long)p->total_tokens > (1LL << 40)) return KVCRUSH_ERR_UNSUPPORTED;
+  s->n_layers = p->n_layers; s->n_seqs = p->n_seqs; s->Hq = p->n_q_heads; s->Hkv = p->n_kv_heads;
+  s->D = p->head_dim; s->T = p->total_tokens; s->max_seqlen = p->max_seqlen; s->causal = p->causal != 0;
+  s->G = p->n_q_heads / p->n_kv_heads; s->W = (p->n_q_heads + 31) / 32;
+  s->cu_seqlens = p->cu_seqlens_dev;
+  return KVCRUSH_OK;
+}
+
+int make_view(const kvcrush_tensor_t* t, int head_dim, TensorView* v) {
+  if (!t || !t->ptr_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if (t->dtype != KVCRUSH_BF16 && t->dtype != KVCRUSH_FP16 && t->dtype != KVCRUSH_FP32) return KVCRUSH_ERR_INVALID_ARG;
+  const int eb = elt_bytes(t->dtype);
+  if (reinterpret_cast<uintptr_t>(t->ptr_dev) % 16 != 0) return KVCRUSH_ERR_MISALIGNED;
+  if ((t->stride_layer * eb) % 16 || (t->stride_token * eb) % 16 || (t->stride_head * eb) % 16 ||
+      ((long long)head_dim * eb) % 16)
+    return KVCRUSH_ERR_MISALIGNED;
+  if (t->stride_layer < 0 || t->stride_token < 0 || t->stride_head < 0) return KVCRUSH_ERR_INVALID_ARG;
+  v->ptr = t->ptr_dev; v->dtype = t->dtype; v->sl = t->stride_layer; v->st = t->stride_token; v->sh = t->stride_head;
+  return KVCRUSH_OK;
+}
+
+size_t score_ws(const Shape& s) { return round_up((size_t)s.n_layers * s.Hq * s.T * sizeof(float)); }
+size_t signature_ws(const Shape& s) { return round_up((size_t)s.n_layers * s.n_seqs * s.Hq * sizeof(float)); }
+
+}  // namespace
+
+extern "C" {
+
+int kvcrush_workspace_size(const kvcrush_problem_t* problem, int stage, size_t* bytes) {
+  Shape s;
+  if (!bytes) return KVCRUSH_ERR_INVALID_ARG;
+  const int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  switch (stage) {
+    case KVCRUSH_STAGE_SCORE: *bytes = score_ws(s); return KVCRUSH_OK;
+    case KVCRUSH_STAGE_SIGNATURE: *bytes = signature_ws(s); return KVCRUSH_OK;
+    case KVCRUSH_STAGE_SELECT: *bytes = select_workspace_bytes(s); return KVCRUSH_OK;
+    case KVCRUSH_STAGE_COMPACT: *bytes = 0; return KVCRUSH_OK;
+    default: return KVCRUSH_ERR_INVALID_ARG;
+  }
+}
+
+int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, const kvcrush_tensor_t* K,
+                  const float* lse_in_dev, float* scores_dev, float* lse_out_dev, int normalize, int impl,
+                  void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  Shape s;
+  int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  TensorView q, k;
+  if ((rc = make_view(Q, s.D, &q)) != KVCRUSH_OK) return rc;
+  if ((rc = make_view(K, s.D, &k)) != KVCRUSH_OK) return rc;
+  if (!scores_dev || !status_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if (q.dtype != k.dtype) return KVCRUSH_ERR_INVALID_ARG;
+  if (q.dtype != KVCRUSH_BF16 && q.dtype != KVCRUSH_FP32) return KVCRUSH_ERR_UNSUPPORTED;
+  if (impl != KVCRUSH_SCORE_AUTO && impl != KVCRUSH_SCORE_SIMT && impl != KVCRUSH_SCORE_TENSOR)
+    return KVCRUSH_ERR_INVALID_ARG;
+  float* lse2_ws = nullptr;
+  if (!lse_in_dev) {
+    if (!workspace || workspace_bytes < score_ws(s)) return KVCRUSH_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
+    lse2_ws = static_cast<float*>(workspace);
+  }
+  const float scale = problem->softmax_scale != 0.f ? problem->softmax_scale : 1.f / sqrtf((float)s.D);
+  const float log2e = 1.4426950408889634f;
+  const float scale_log2 = scale * log2e;
+  const bool tensor_ok = score_tensor_supported(s, q, k);
+  if (impl == KVCRUSH_SCORE_TENSOR && !tensor_ok) return KVCRUSH_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (impl == KVCRUSH_SCORE_SIMT || !tensor_ok)
+    return launch_score_simt(s, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, scores_dev, lse_out_dev, normalize,
+                             status_dev, st);
+  return launch_score_tensor(s, problem->cu_seqlens_host, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, scores_dev,
+                             lse_out_dev, normalize, status_dev, st);
+}
+
+int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev, const int32_t* sig_keep_dev,
+                      const float* theta_in_dev, uint32_t* sigs_dev, float* theta_out_dev,
+                      void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  Shape s;
+  const int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if (!scores_dev || !sigs_dev || !status_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if (!theta_in_dev && !sig_keep_dev) return KVCRUSH_ERR_INVALID_ARG;
+  float* theta = theta_out_dev;
+  if (!theta_in_dev && !theta) {
+    if (!workspace || workspace_bytes < signature_ws(s)) return KVCRUSH_ERR_WORKSPACE;
+    theta = static_cast<float*>(workspace);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (theta_in_dev && theta_out_dev && theta_out_dev != theta_in_dev) {
+    if (cudaMemcpyAsync(theta_out_dev, theta_in_dev, (size_t)s.n_layers * s.n_seqs * s.Hq * sizeof(float),
+                        cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return KVCRUSH_ERR_CUDA;
+  }
+  return launch_signature(s, scores_dev, sig_keep_dev, theta_in_dev, sigs_dev, theta, st);
+}
+
+int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
+                   const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                   const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev,
+                   void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  Shape s;
+  const int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if (!scores_dev || !sigs_dev || !budget_imp_dev || !budget_rep_dev || !cu_kept_dev || !idx_dev || !status_dev)
+    return KVCRUSH_ERR_INVALID_ARG;
+  if (anchor_mode != KVCRUSH_ANCHOR_ALTERNATE && anchor_mode != KVCRUSH_ANCHOR_MEAN &&
+      anchor_mode != KVCRUSH_ANCHOR_EXPLICIT)
+    return KVCRUSH_ERR_INVALID_ARG;
+  if (anchor_mode == KVCRUSH_ANCHOR_EXPLICIT && !anchor_bits_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if (s.max_seqlen > 262144) return KVCRUSH_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < select_workspace_bytes(s)) return KVCRUSH_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
+  return launch_select(s, scores_dev, sigs_dev, budget_imp_dev, budget_rep_dev, anchor_mode, anchor_bits_dev,
+                       anchor_per_segment != 0, cu_kept_dev, idx_dev, kind_dev, workspace,
+                       static_cast<cudaStream_t>(stream));
+}
+
+int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K, const kvcrush_tensor_t* V,
+                    const int32_t* cu_kept_dev, const int32_t* idx_dev, int64_t total_kept,
+                    const kvcrush_tensor_t* K_out, const kvcrush_tensor_t* V_out,
+                    int32_t* status_dev, void* stream) {
+  Shape s;
+  int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if (!cu_kept_dev || !idx_dev || !status_dev || total_kept < 0) return KVCRUSH_ERR_INVALID_ARG;
+  if ((V == nullptr) != (V_out == nullptr)) return KVCRUSH_ERR_INVALID_ARG;
+  TensorView k, v, ko, vo;
+  if ((rc = make_view(K, s.D, &k)) != KVCRUSH_OK) return rc;
+  if ((rc = make_view(K_out, s.D, &ko)) != KVCRUSH_OK) return rc;
+  if (k.dtype != ko.dtype) return KVCRUSH_ERR_INVALID_ARG;
+  if (V) {
+    if ((rc = make_view(V, s.D, &v)) != KVCRUSH_OK) return rc;
+    if ((rc = make_view(V_out, s.D, &vo)) != KVCRUSH_OK) return rc;
+    if (v.dtype != k.dtype || vo.dtype != k.dtype) return KVCRUSH_ERR_INVALID_ARG;
+  }
+  return launch_compact(s, k, V ? &v : nullptr, cu_kept_dev, idx_dev, total_kept, ko, V ? &vo : nullptr,
+                        static_cast<cudaStream_t>(stream));
+}
+
+const char* kvcrush_strerror(int code) {
+  switch (code) {
+    case KVCRUSH_OK: return "ok";
+    case KVCRUSH_ERR_INVALID_ARG: return "invalid argument";
+    case KVCRUSH_ERR_UNSUPPORTED: return "unsupported shape or type";
+    case KVCRUSH_ERR_MISALIGNED: return "misaligned pointer or stride";
+    case KVCRUSH_ERR_WORKSPACE: return "workspace missing or too small";
+    case KVCRUSH_ERR_CUDA: return "CUDA call failed";
+    default: return "unknown error";
+  }
+}
+
+int kvcrush_version(void) { return 100; }
+
+}  // extern "C"

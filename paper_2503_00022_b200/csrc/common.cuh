@@ -1,0 +1,74 @@
+// Shared declarations of the kvcrush CUDA library (internal; the public ABI is include/kvcrush.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvcrush.h"
+
+namespace kvc {
+
+// Device-side view of the problem shape, passed by value to every kernel.
+struct Shape {
+  int n_layers, n_seqs, Hq, Hkv, D, T, max_seqlen, causal;
+  int G;                       // Hq / Hkv
+  int W;                       // signature words per token
+  const int32_t* cu_seqlens;   // device, [n_seqs + 1]
+};
+
+struct TensorView {
+  const void* ptr;
+  int dtype;
+  long long sl, st, sh;        // strides in elements: layer, token, head
+};
+
+inline int elt_bytes(int dtype) { return dtype == KVCRUSH_FP32 ? 4 : 2; }
+
+// kernel ids written to status[1]
+enum KernelId { KID_SCORE_LSE = 1, KID_SCORE_COLSUM = 2 };
+
+__device__ __forceinline__ void report(int32_t* status, int code, int kid, int a, int b) {
+  if (atomicCAS(status, 0, code) == 0) {
+    status[1] = kid;
+    status[2] = a;
+    status[3] = b;
+  }
+}
+
+// Sequence that owns packed token `tok` (binary search in cu_seqlens).
+__device__ __forceinline__ int seq_of_token(const int32_t* __restrict__ cu, int n_seqs, int tok) {
+  int lo = 0, hi = n_seqs;          // invariant: cu[lo] <= tok < cu[hi]
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (__ldg(cu + mid) <= tok) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// ---- stage launchers (defined in the per-stage .cu files) -------------------------------------------
+
+// score: SIMT fp32 kernels (any dtype/shape) and tcgen05 kernels (bf16, D in {64,128}).
+// lse2_ws: [n_layers][Hq][T] float32 row log-sum-exp in the log2 domain (written unless lse_in is given).
+int launch_score_simt(const Shape& s, const TensorView& Q, const TensorView& K, float scale_log2,
+                      const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores, float* lse_out,
+                      int normalize, int32_t* status, cudaStream_t stream);
+bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorView& K);
+int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView& Q, const TensorView& K,
+                        float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores,
+                        float* lse_out, int normalize, int32_t* status, cudaStream_t stream);
+
+int launch_signature(const Shape& s, const float* scores, const int32_t* sig_keep, const float* theta_in,
+                     uint32_t* sigs, float* theta, cudaStream_t stream);
+
+size_t select_workspace_bytes(const Shape& s);
+int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, const int32_t* budget_imp,
+                  const int32_t* budget_rep, int anchor_mode, const uint32_t* anchor_bits, int anchor_per_segment,
+                  const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws, cudaStream_t stream);
+
+int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, const int32_t* cu_kept,
+                   const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,
+                   cudaStream_t stream);
+
+inline int check_launch() { return cudaGetLastError() == cudaSuccess ? KVCRUSH_OK : KVCRUSH_ERR_CUDA; }
+
+}  // namespace kvc

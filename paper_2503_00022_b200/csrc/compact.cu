@@ -1,0 +1,95 @@
+// Stage 4: gather of the kept K/V rows into the reduced cache (Sec. 3.2 of the paper: the
+// representatives together with the important tokens form the final cache).
+//
+// Pure byte movement, bound by HBM bandwidth.  One warp owns one kept token of one layer and
+// copies that token's rows of every KV head, for K and for V, as 16-byte vectors: the index
+// arithmetic (segment search, source token) is paid once per token, and every lane keeps four
+// independent 16-byte loads in flight before the first store.
+#include "common.cuh"
+
+namespace kvc {
+
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+
+struct CompactArgs {
+  const unsigned char* src[2];
+  unsigned char* dst[2];
+  long long src_sl[2], src_st[2], src_sh[2];   // bytes
+  long long dst_sl[2], dst_st[2], dst_sh[2];   // bytes
+  int n_tensors;
+  int vec_per_row;                             // 16-byte vectors in one head row
+  int n_vec;                                   // vectors per token = Hkv * vec_per_row
+};
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+compact_kernel(Shape s, CompactArgs a, const int32_t* __restrict__ cu_kept, const int32_t* __restrict__ idx,
+               long long total_kept) {
+  const int lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  if (row >= total_kept) return;
+
+  // segment = layer * n_seqs + seq that owns kept row `row`
+  const int n_seg = s.n_layers * s.n_seqs;
+  int lo = 0, hi = n_seg;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if ((long long)__ldg(cu_kept + mid) <= row) lo = mid; else hi = mid;
+  }
+  const int layer = lo / s.n_seqs, seq = lo - layer * s.n_seqs;
+  const long long src_tok = (long long)__ldg(s.cu_seqlens + seq) + __ldg(idx + row);
+  const long long dst_tok = row - __ldg(cu_kept + layer * s.n_seqs);
+
+#pragma unroll 1
+  for (int ten = 0; ten < a.n_tensors; ++ten) {
+    const unsigned char* sp = a.src[ten] + layer * a.src_sl[ten] + src_tok * a.src_st[ten];
+    unsigned char* dp = a.dst[ten] + layer * a.dst_sl[ten] + dst_tok * a.dst_st[ten];
+    for (int v0 = lane; v0 < a.n_vec; v0 += 4 * 32) {
+      uint4 val[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + u * 32;
+        if (v < a.n_vec) {
+          const int h = v / a.vec_per_row, c = v - h * a.vec_per_row;
+          val[u] = __ldcs(reinterpret_cast<const uint4*>(sp + h * a.src_sh[ten]) + c);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + u * 32;
+        if (v < a.n_vec) {
+          const int h = v / a.vec_per_row, c = v - h * a.vec_per_row;
+          __stcs(reinterpret_cast<uint4*>(dp + h * a.dst_sh[ten]) + c, val[u]);
+        }
+      }
+    }
+  }
+}
+
+}  // namespace
+
+int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, const int32_t* cu_kept,
+                   const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,
+                   cudaStream_t stream) {
+  if (total_kept == 0) return KVCRUSH_OK;
+  const int eb = elt_bytes(K.dtype);
+  CompactArgs a{};
+  a.n_tensors = V ? 2 : 1;
+  const TensorView* in[2] = {&K, V};
+  const TensorView* out[2] = {&K_out, V_out};
+  for (int i = 0; i < a.n_tensors; ++i) {
+    a.src[i] = static_cast<const unsigned char*>(in[i]->ptr);
+    a.dst[i] = static_cast<unsigned char*>(const_cast<void*>(out[i]->ptr));
+    a.src_sl[i] = in[i]->sl * eb; a.src_st[i] = in[i]->st * eb; a.src_sh[i] = in[i]->sh * eb;
+    a.dst_sl[i] = out[i]->sl * eb; a.dst_st[i] = out[i]->st * eb; a.dst_sh[i] = out[i]->sh * eb;
+  }
+  a.vec_per_row = s.D * eb / 16;
+  a.n_vec = s.Hkv * a.vec_per_row;
+  const long long blocks = (total_kept + kWarpsPerBlock - 1) / kWarpsPerBlock;
+  if (blocks > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
+  compact_kernel<<<(unsigned)blocks, kWarpsPerBlock * 32, 0, stream>>>(s, a, cu_kept, idx, total_kept);
+  return check_launch();
+}
+
+}  // namespace kvc

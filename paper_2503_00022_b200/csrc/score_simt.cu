@@ -1,0 +1,165 @@
+// Stage 1 on CUDA cores (fp32 arithmetic): attention column sums (Algorithm 1 of the paper,
+// "attention weights" and "normalized attention score" steps).  Serves fp32 inputs and shapes the
+// tensor-core kernels do not cover; the S x S matrix is never stored.
+//
+//   lse_rows_kernel   one warp per query row j: lanes take keys t, t+32, ..; each lane keeps an
+//                     online (max, sum) pair in the log2 domain; lse2(j) = log2 sum_t 2^(s2(j,t))
+//                     with s2 = q.k * scale * log2(e).
+//   colsum_kernel     one warp per key t: lanes take queries j, j+32, ..; accumulates
+//                     2^(s2(j,t) - lse2(j)) = A(j,t) and reduces over the warp.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace kvc {
+
+namespace {
+
+constexpr int kWarpsPerBlock = 4;
+constexpr int kMaxD = 256;
+
+template <typename T>
+__device__ __forceinline__ void load8(const T* p, float (&v)[8]);
+
+template <>
+__device__ __forceinline__ void load8<float>(const float* p, float (&v)[8]) {
+  const float4 a = __ldg(reinterpret_cast<const float4*>(p));
+  const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+template <>
+__device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ float dot_row(const float* __restrict__ a_sh, const T* __restrict__ b, int D) {
+  float acc = 0.f;
+  for (int d = 0; d < D; d += 8) {
+    float v[8];
+    load8<T>(b + d, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc = fmaf(a_sh[d + i], v[i], acc);
+  }
+  return acc;
+}
+
+template <typename T>
+__device__ __forceinline__ void stage_row(float* sh, const T* row, int D, int lane) {
+  for (int d = lane * 8; d < D; d += 32 * 8) {
+    float v[8];
+    load8<T>(row + d, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sh[d + i] = v[i];
+  }
+  __syncwarp();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+lse_rows_kernel(Shape s, TensorView Q, TensorView K, float scale_log2, float* __restrict__ lse2,
+                float* __restrict__ lse_out) {
+  __shared__ float q_sh[kWarpsPerBlock][kMaxD];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const long long row = (long long)blockIdx.x * kWarpsPerBlock + wib;     // (layer, head, token)
+  if (row >= (long long)s.n_layers * s.Hq * s.T) return;
+  const int tok = (int)(row % s.T);
+  const int h = (int)((row / s.T) % s.Hq);
+  const int layer = (int)(row / ((long long)s.T * s.Hq));
+  const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
+  const int t0 = __ldg(s.cu_seqlens + seq), t1 = __ldg(s.cu_seqlens + seq + 1);
+  const int t_end = s.causal ? tok + 1 : t1;
+
+  const T* q = static_cast<const T*>(Q.ptr) + layer * Q.sl + (long long)tok * Q.st + h * Q.sh;
+  const T* kbase = static_cast<const T*>(K.ptr) + layer * K.sl + (h / s.G) * K.sh;
+  stage_row<T>(q_sh[wib], q, s.D, lane);
+
+  float m = -INFINITY, sum = 0.f;
+  for (int t = t0 + lane; t < t_end; t += 32) {
+    const float x = dot_row<T>(q_sh[wib], kbase + (long long)t * K.st, s.D) * scale_log2;
+    if (x > m) { sum = sum * exp2f(m - x) + 1.f; m = x; } else { sum += exp2f(x - m); }
+  }
+  float big = m;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) big = fmaxf(big, __shfl_xor_sync(0xFFFFFFFFu, big, d));
+  float part = (m == -INFINITY) ? 0.f : sum * exp2f(m - big);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, d);
+  if (lane == 0) {
+    const float v = big + log2f(part);
+    lse2[row] = v;
+    if (lse_out) lse_out[row] = v * 0.69314718055994530942f;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+colsum_kernel(Shape s, TensorView Q, TensorView K, float scale_log2, const float* __restrict__ lse,
+              float lse_mul, float* __restrict__ scores, int normalize) {
+  __shared__ float k_sh[kWarpsPerBlock][kMaxD];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const long long col = (long long)blockIdx.x * kWarpsPerBlock + wib;     // (layer, head, token)
+  if (col >= (long long)s.n_layers * s.Hq * s.T) return;
+  const int tok = (int)(col % s.T);
+  const int h = (int)((col / s.T) % s.Hq);
+  const int layer = (int)(col / ((long long)s.T * s.Hq));
+  const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
+  const int t0 = __ldg(s.cu_seqlens + seq), t1 = __ldg(s.cu_seqlens + seq + 1);
+  const int j_begin = s.causal ? tok : t0;
+
+  const T* k = static_cast<const T*>(K.ptr) + layer * K.sl + (long long)tok * K.st + (h / s.G) * K.sh;
+  const T* qbase = static_cast<const T*>(Q.ptr) + layer * Q.sl + h * Q.sh;
+  const float* lse_row = lse + ((long long)layer * s.Hq + h) * s.T;
+  stage_row<T>(k_sh[wib], k, s.D, lane);
+
+  float acc = 0.f;
+  for (int j = j_begin + lane; j < t1; j += 32) {
+    const float x = dot_row<T>(k_sh[wib], qbase + (long long)j * Q.st, s.D) * scale_log2;
+    acc += exp2f(x - __ldg(lse_row + j) * lse_mul);
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, d);
+  if (lane == 0) scores[col] = normalize ? acc / (float)(t1 - t0) : acc;
+}
+
+template <typename T>
+int run(const Shape& s, const TensorView& Q, const TensorView& K, float scale_log2, const float* lse_in,
+        float lse_in_mul, float* lse2_ws, float* scores, float* lse_out, int normalize, cudaStream_t stream) {
+  const long long rows = (long long)s.n_layers * s.Hq * s.T;
+  if (rows == 0) return KVCRUSH_OK;
+  const long long blocks = (rows + kWarpsPerBlock - 1) / kWarpsPerBlock;
+  if (blocks > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
+  const float* lse = lse_in;
+  float mul = lse_in_mul;
+  if (!lse_in) {
+    lse_rows_kernel<T><<<(unsigned)blocks, kWarpsPerBlock * 32, 0, stream>>>(s, Q, K, scale_log2, lse2_ws, lse_out);
+    if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+    lse = lse2_ws;
+    mul = 1.f;
+  }
+  colsum_kernel<T><<<(unsigned)blocks, kWarpsPerBlock * 32, 0, stream>>>(s, Q, K, scale_log2, lse, mul, scores,
+                                                                          normalize);
+  return check_launch();
+}
+
+}  // namespace
+
+int launch_score_simt(const Shape& s, const TensorView& Q, const TensorView& K, float scale_log2,
+                      const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores, float* lse_out,
+                      int normalize, int32_t* /*status*/, cudaStream_t stream) {
+  if (s.D > kMaxD || s.D % 8 != 0) return KVCRUSH_ERR_UNSUPPORTED;
+  if (Q.dtype == KVCRUSH_FP32)
+    return run<float>(s, Q, K, scale_log2, lse_in, lse_in_mul, lse2_ws, scores, lse_out, normalize, stream);
+  if (Q.dtype == KVCRUSH_BF16)
+    return run<__nv_bfloat16>(s, Q, K, scale_log2, lse_in, lse_in_mul, lse2_ws, scores, lse_out, normalize, stream);
+  return KVCRUSH_ERR_UNSUPPORTED;
+}
+
+}  // namespace kvc

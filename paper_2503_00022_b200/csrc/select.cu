@@ -1,0 +1,397 @@
+// Stage 3: the kept set of every (layer, sequence) segment (Sec. 3 and Algorithm 2 of the paper).
+//
+//   importance_kernel      I(t) = sum of the per-head scores of token t (H2O's cumulative attention),
+//                          float64, heads added in ascending order inside each KV group and the
+//                          group sums added in ascending order; stored as an order-preserving
+//                          64-bit key.  One thread per (layer, token), coalesced per-head rows.
+//   select_segment_kernel  one CTA per segment:
+//                            1. exact radix select of the B_imp-th largest key, ties admitted in
+//                               ascending token order                         -> important set
+//                            2. anchor; d_t = popc(sig_t xor anchor) for the other tokens
+//                            3. stable counting sort by (d_t, t): every warp owns a contiguous
+//                               token range, per-warp histograms, one scan, ordered scatter
+//                            4. equal-frequency buckets of the sorted order; per bucket the member
+//                               minimising  sum_{h: bit set} (m - 2 n_h)  (= L1 distance to the
+//                               per-bit mean, up to a constant), ties to the lower token
+//                            5. kept = important U representatives, ascending token index
+// All decisions are integer or exact float64 comparisons, so the result is unique.
+#include "common.cuh"
+
+namespace kvc {
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxBins = 129;              // Hamming distances 0..128
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+__global__ void __launch_bounds__(256)
+importance_kernel(Shape s, const float* __restrict__ scores, unsigned long long* __restrict__ keys) {
+  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= (long long)s.n_layers * s.T) return;
+  const int layer = (int)(gid / s.T), tok = (int)(gid - (long long)layer * s.T);
+  const float* sc = scores + (size_t)layer * s.Hq * s.T + tok;
+  double total = 0.0;
+  for (int g = 0; g < s.Hkv; ++g) {
+    double group = 0.0;
+    for (int j = 0; j < s.G; ++j)
+      group = __dadd_rn(group, (double)__ldg(sc + (size_t)(g * s.G + j) * s.T));
+    total = __dadd_rn(total, group);
+  }
+  total = __dadd_rn(total, 0.0);           // -0.0 -> +0.0
+  const unsigned long long b = (unsigned long long)__double_as_longlong(total);
+  keys[gid] = (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+}
+
+struct SelectArgs {
+  const unsigned long long* keys;     // [n_layers][T]
+  const uint32_t* sigs;               // [n_layers][T][W]
+  const int32_t* budget_imp;
+  const int32_t* budget_rep;
+  int anchor_mode;
+  const uint32_t* anchor_bits;
+  int anchor_per_segment;
+  const int32_t* cu_kept;
+  int32_t* idx;
+  uint8_t* kind;
+  int32_t* sorted;                    // [n_layers][T] scratch: grouped tokens in (d, t) order
+  int mask_words;                     // words of one membership mask in shared memory
+};
+
+__device__ __forceinline__ uint32_t head_mask(int Hq, int w) {
+  const int n = Hq - 32 * w;
+  return n >= 32 ? 0xFFFFFFFFu : ((1u << n) - 1u);
+}
+
+__global__ void __launch_bounds__(kThreads)
+select_segment_kernel(Shape s, SelectArgs a) {
+  extern __shared__ uint32_t dyn_smem[];
+  uint32_t* imp_mask = dyn_smem;
+  uint32_t* rep_mask = dyn_smem + a.mask_words;
+
+  __shared__ uint32_t hist[256];
+  __shared__ unsigned long long sel_prefix;
+  __shared__ uint32_t sel_k;
+  __shared__ int warp_hist[kWarps][kMaxBins];
+  __shared__ int bin_base[kMaxBins + 1];
+  __shared__ int warp_tot[kWarps];
+  __shared__ int bit_cnt[128];
+  __shared__ uint32_t anchor_sh[4];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned lt_mask = (1u << lane) - 1u;
+  const int seg = blockIdx.x;
+  const int layer = seg / s.n_seqs, seq = seg - layer * s.n_seqs;
+  const int t0 = __ldg(s.cu_seqlens + seq);
+  const int L = __ldg(s.cu_seqlens + seq + 1) - t0;
+  const int b_imp = max(0, __ldg(a.budget_imp + seg));
+  const int b_rep = max(0, __ldg(a.budget_rep + seg));
+  int32_t* out_idx = a.idx + __ldg(a.cu_kept + seg);
+  uint8_t* out_kind = a.kind ? a.kind + __ldg(a.cu_kept + seg) : nullptr;
+
+  if ((long long)b_imp + b_rep >= L) {             // budget covers the sequence: keep everything
+    for (int i = tid; i < L; i += kThreads) {
+      out_idx[i] = i;
+      if (out_kind) out_kind[i] = 0;
+    }
+    return;
+  }
+
+  const unsigned long long* keys = a.keys + (size_t)layer * s.T + t0;
+  const uint32_t* sig = a.sigs + ((size_t)layer * s.T + t0) * s.W;
+  int32_t* sorted = a.sorted + (size_t)layer * s.T + t0;
+  const int n_words = (L + 31) >> 5;
+  // contiguous token range of this warp (multiple of 32 tokens so that mask words do not straddle)
+  const int per_warp = ((n_words + kWarps - 1) / kWarps) * 32;
+  const int r_lo = min(L, warp * per_warp), r_hi = min(L, r_lo + per_warp);
+
+  for (int i = tid; i < n_words; i += kThreads) { imp_mask[i] = 0; rep_mask[i] = 0; }
+  __syncthreads();
+
+  // ---- 1. important tokens: the b_imp largest keys, ties to the lower index --------------------
+  if (b_imp > 0) {
+    unsigned long long prefix = 0;
+    uint32_t k_rem = b_imp;
+    for (int shift = 56; shift >= 0; shift -= 8) {
+      for (int i = tid; i < 256; i += kThreads) hist[i] = 0;
+      __syncthreads();
+      const unsigned long long hi_mask = shift == 56 ? 0ull : (~0ull << (shift + 8));
+      for (int base = 0; base < L; base += kThreads) {
+        const int i = base + tid;
+        const bool in = i < L;
+        const unsigned long long key = in ? __ldg(keys + i) : 0ull;
+        const bool live = in && ((key & hi_mask) == prefix);
+        const uint32_t digit = (uint32_t)(key >> shift) & 0xFFu;
+        const unsigned voters = __ballot_sync(kFull, live);
+        if (live) {
+          const unsigned peers = __match_any_sync(voters, digit);
+          if ((peers & lt_mask) == 0) atomicAdd(&hist[digit], __popc(peers));
+        }
+      }
+      __syncthreads();
+      if (warp == 0) {
+        uint32_t local = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) local += hist[255 - 8 * lane - j];
+        uint32_t incl = local;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t v = __shfl_up_sync(kFull, incl, d);
+          if (lane >= d) incl += v;
+        }
+        const uint32_t excl = incl - local;
+        if (excl < k_rem && k_rem <= incl) {
+          uint32_t acc = excl;
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t c = hist[255 - 8 * lane - j];
+            if (k_rem <= acc + c) {
+              sel_prefix = prefix | ((unsigned long long)(255 - 8 * lane - j) << shift);
+              sel_k = k_rem - acc;
+              break;
+            }
+            acc += c;
+          }
+        }
+      }
+      __syncthreads();
+      prefix = sel_prefix;
+      k_rem = sel_k;
+      __syncthreads();
+    }
+    // prefix = the b_imp-th largest key; k_rem = how many keys equal to it are admitted
+    const unsigned long long kth = prefix;
+    int n_eq = 0;
+    for (int i = r_lo + lane; i < r_hi; i += 32) n_eq += (__ldg(keys + i) == kth);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) n_eq += __shfl_xor_sync(kFull, n_eq, d);
+    if (lane == 0) warp_tot[warp] = n_eq;
+    __syncthreads();
+    int eq_before = 0;
+    for (int w = 0; w < warp; ++w) eq_before += warp_tot[w];
+    for (int base = r_lo; base < r_hi; base += 32) {
+      const int i = base + lane;
+      const unsigned long long key = i < r_hi ? __ldg(keys + i) : 0ull;
+      const bool eq = i < r_hi && key == kth;
+      const unsigned eq_b = __ballot_sync(kFull, eq);
+      const bool imp = i < r_hi && (key > kth || (eq && (uint32_t)(eq_before + __popc(eq_b & lt_mask)) < k_rem));
+      const unsigned imp_b = __ballot_sync(kFull, imp);
+      if (lane == 0) imp_mask[base >> 5] = imp_b;
+      eq_before += __popc(eq_b);
+    }
+    __syncthreads();
+  }
+
+  // ---- 2-4. representatives of the other tokens ------------------------------------------------
+  if (b_rep > 0) {
+    const int N = L - b_imp;
+    const int W = s.W;
+    // anchor
+    if (a.anchor_mode == KVCRUSH_ANCHOR_MEAN) {
+      for (int i = tid; i < 128; i += kThreads) bit_cnt[i] = 0;
+      __syncthreads();
+      int acc[4] = {0, 0, 0, 0};
+      for (int base = r_lo; base < r_hi; base += 32) {
+        const int i = base + lane;
+        const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
+        for (int w = 0; w < W; ++w) {
+          const uint32_t word = cand ? __ldg(sig + (size_t)i * W + w) : 0u;
+          const int nb = min(32, s.Hq - 32 * w);
+          for (int b = 0; b < nb; ++b) {
+            const unsigned m = __ballot_sync(kFull, (word >> b) & 1u);
+            if (lane == b) acc[w] += __popc(m);
+          }
+        }
+      }
+      for (int w = 0; w < W; ++w)
+        if (32 * w + lane < s.Hq && acc[w]) atomicAdd(&bit_cnt[32 * w + lane], acc[w]);
+      __syncthreads();
+      if (warp < W) {
+        const int h = 32 * warp + lane;
+        const unsigned word = __ballot_sync(kFull, h < s.Hq && 2LL * bit_cnt[h] >= N);
+        if (lane == 0) anchor_sh[warp] = word;
+      }
+    } else if (tid < W) {
+      uint32_t word;
+      if (a.anchor_mode == KVCRUSH_ANCHOR_EXPLICIT)
+        word = __ldg(a.anchor_bits + (a.anchor_per_segment ? (size_t)seg * W : 0) + tid);
+      else
+        word = 0xAAAAAAAAu;
+      anchor_sh[tid] = word & head_mask(s.Hq, tid);
+    }
+    for (int i = tid; i < kWarps * kMaxBins; i += kThreads) (&warp_hist[0][0])[i] = 0;
+    __syncthreads();
+    uint32_t anc[4], hm[4];
+    for (int w = 0; w < 4; ++w) { anc[w] = w < W ? anchor_sh[w] : 0u; hm[w] = w < W ? head_mask(s.Hq, w) : 0u; }
+    const int n_bins = s.Hq + 1;
+
+    // counting sort by (d, t): per-warp histograms over contiguous token ranges
+    for (int base = r_lo; base < r_hi; base += 32) {
+      const int i = base + lane;
+      const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
+      int d = 0;
+      if (cand)
+        for (int w = 0; w < W; ++w) d += __popc((__ldg(sig + (size_t)i * W + w) ^ anc[w]) & hm[w]);
+      const unsigned voters = __ballot_sync(kFull, cand);
+      if (cand) {
+        const unsigned peers = __match_any_sync(voters, d);
+        if ((peers & lt_mask) == 0) warp_hist[warp][d] += __popc(peers);
+      }
+      __syncwarp();
+    }
+    __syncthreads();
+    if (tid < n_bins) {                     // per bin: exclusive prefix over warps (token order)
+      int run = 0;
+      for (int w = 0; w < kWarps; ++w) { const int c = warp_hist[w][tid]; warp_hist[w][tid] = run; run += c; }
+      bin_base[tid + 1] = run;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      bin_base[0] = 0;
+      for (int b = 1; b <= n_bins; ++b) bin_base[b] += bin_base[b - 1];
+    }
+    __syncthreads();
+    for (int base = r_lo; base < r_hi; base += 32) {
+      const int i = base + lane;
+      const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
+      int d = 0;
+      if (cand)
+        for (int w = 0; w < W; ++w) d += __popc((__ldg(sig + (size_t)i * W + w) ^ anc[w]) & hm[w]);
+      const unsigned voters = __ballot_sync(kFull, cand);
+      unsigned peers = 0;
+      if (cand) {
+        peers = __match_any_sync(voters, d);
+        sorted[bin_base[d] + warp_hist[warp][d] + __popc(peers & lt_mask)] = i;
+      }
+      __syncwarp();
+      if (cand && (peers & lt_mask) == 0) warp_hist[warp][d] += __popc(peers);
+      __syncwarp();
+    }
+    __syncthreads();
+
+    // one representative per equal-frequency bucket (one warp per bucket)
+    for (int bkt = warp; bkt < b_rep; bkt += kWarps) {
+      const int lo = (int)(((long long)bkt * N) / b_rep);
+      const int hi = (int)(((long long)(bkt + 1) * N) / b_rep);
+      const int m = hi - lo;
+      unsigned long long best = ~0ull;
+      if (m <= 32) {
+        const bool member = lane < m;
+        const int t = member ? sorted[lo + lane] : 0;
+        int cost = 0;
+        for (int w = 0; w < W; ++w) {
+          const uint32_t word = member ? __ldg(sig + (size_t)t * W + w) : 0u;
+          const int nb = min(32, s.Hq - 32 * w);
+          for (int b = 0; b < nb; ++b) {
+            const unsigned ones = __ballot_sync(kFull, (word >> b) & 1u);
+            if ((word >> b) & 1u) cost += m - 2 * __popc(ones);
+          }
+        }
+        if (member) best = ((unsigned long long)((uint32_t)cost + 0x80000000u) << 32) | (uint32_t)t;
+      } else {
+        int n_ones[4] = {0, 0, 0, 0};        // lane b of word w holds n_h for head 32w+b
+        for (int c0 = lo; c0 < hi; c0 += 32) {
+          const bool member = c0 + lane < hi;
+          const int t = member ? sorted[c0 + lane] : 0;
+          for (int w = 0; w < W; ++w) {
+            const uint32_t word = member ? __ldg(sig + (size_t)t * W + w) : 0u;
+            const int nb = min(32, s.Hq - 32 * w);
+            for (int b = 0; b < nb; ++b) {
+              const unsigned ones = __ballot_sync(kFull, (word >> b) & 1u);
+              if (lane == b) n_ones[w] += __popc(ones);
+            }
+          }
+        }
+        for (int c0 = lo; c0 < hi; c0 += 32) {
+          const bool member = c0 + lane < hi;
+          const int t = member ? sorted[c0 + lane] : 0;
+          int cost = 0;
+          for (int w = 0; w < W; ++w) {
+            const uint32_t word = member ? __ldg(sig + (size_t)t * W + w) : 0u;
+            const int nb = min(32, s.Hq - 32 * w);
+            for (int b = 0; b < nb; ++b) {
+              const int n_h = __shfl_sync(kFull, n_ones[w], b);
+              if ((word >> b) & 1u) cost += m - 2 * n_h;
+            }
+          }
+          if (member) {
+            const unsigned long long key = ((unsigned long long)((uint32_t)cost + 0x80000000u) << 32) | (uint32_t)t;
+            best = key < best ? key : best;
+          }
+        }
+      }
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(kFull, best, d);
+        best = o < best ? o : best;
+      }
+      if (lane == 0) {
+        const uint32_t t = (uint32_t)best;
+        atomicOr(&rep_mask[t >> 5], 1u << (t & 31));
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- 5. kept = important U representatives, ascending ------------------------------------------
+  const int wpt = (n_words + kThreads - 1) / kThreads;      // mask words per thread, contiguous
+  const int w_lo = min(n_words, tid * wpt), w_hi = min(n_words, w_lo + wpt);
+  int cnt = 0;
+  for (int w = w_lo; w < w_hi; ++w) cnt += __popc(imp_mask[w] | rep_mask[w]);
+  int incl = cnt;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int v = __shfl_up_sync(kFull, incl, d);
+    if (lane >= d) incl += v;
+  }
+  __syncthreads();                          // warp_tot is reused
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  int pos = incl - cnt;
+  for (int w = 0; w < warp; ++w) pos += warp_tot[w];
+  for (int w = w_lo; w < w_hi; ++w) {
+    const uint32_t rep = rep_mask[w];
+    uint32_t bits = imp_mask[w] | rep;
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      out_idx[pos] = 32 * w + b;
+      if (out_kind) out_kind[pos] = (rep >> b) & 1u;
+      ++pos;
+    }
+  }
+}
+
+}  // namespace
+
+size_t select_workspace_bytes(const Shape& s) {
+  const size_t n = (size_t)s.n_layers * s.T;
+  return ((n * 8 + 255) / 256) * 256 + ((n * 4 + 255) / 256) * 256;
+}
+
+int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, const int32_t* budget_imp,
+                  const int32_t* budget_rep, int anchor_mode, const uint32_t* anchor_bits, int anchor_per_segment,
+                  const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws, cudaStream_t stream) {
+  if (s.T == 0) return KVCRUSH_OK;
+  const size_t n = (size_t)s.n_layers * s.T;
+  unsigned long long* keys = static_cast<unsigned long long*>(ws);
+  int32_t* sorted = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(ws) + ((n * 8 + 255) / 256) * 256);
+  importance_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, scores, keys);
+  if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+
+  SelectArgs a{};
+  a.keys = keys; a.sigs = sigs; a.budget_imp = budget_imp; a.budget_rep = budget_rep;
+  a.anchor_mode = anchor_mode; a.anchor_bits = anchor_bits; a.anchor_per_segment = anchor_per_segment;
+  a.cu_kept = cu_kept; a.idx = idx; a.kind = kind; a.sorted = sorted;
+  a.mask_words = ((s.max_seqlen + 31) / 32 + 3) & ~3;
+  const size_t dyn = (size_t)a.mask_words * 2 * sizeof(uint32_t);
+  if (dyn > 16 * 1024) {     // static + dynamic shared memory above the 48 KB default needs the opt-in
+    if (cudaFuncSetAttribute(select_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) !=
+        cudaSuccess)
+      return KVCRUSH_ERR_CUDA;
+  }
+  select_segment_kernel<<<(unsigned)(s.n_layers * s.n_seqs), kThreads, dyn, stream>>>(s, a);
+  return check_launch();
+}
+
+}  // namespace kvc

@@ -1,0 +1,136 @@
+// Stage 2: per-head thresholds and packed binary signatures (Algorithm 1 and Sec. 3.1 of the paper).
+//
+//   theta_select_kernel   theta = keep-th largest score of one (layer, sequence, head): an exact
+//                         MSB-first radix select over order-preserving 32-bit keys (4 sweeps of 8
+//                         bits, warp-aggregated shared-memory histograms).
+//   binarise_pack_kernel  one thread per (layer, token): compares the token's score of every head
+//                         with that head's threshold and packs the bits.  Lanes are consecutive
+//                         tokens, so every per-head load is a coalesced 128-byte row.
+#include "common.cuh"
+
+namespace kvc {
+
+namespace {
+
+constexpr int kSelectThreads = 512;
+
+// float -> uint32 such that a < b  <=>  key(a) < key(b) (for non-NaN values)
+__device__ __forceinline__ uint32_t order_key(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_to_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+__global__ void __launch_bounds__(kSelectThreads)
+theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __restrict__ sig_keep,
+                    float* __restrict__ theta) {
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t sel_prefix, sel_k;
+
+  const int h = blockIdx.x % s.Hq;
+  const int seg = blockIdx.x / s.Hq;              // layer * n_seqs + seq
+  const int layer = seg / s.n_seqs, seq = seg - layer * s.n_seqs;
+  const int t0 = __ldg(s.cu_seqlens + seq);
+  const int L = __ldg(s.cu_seqlens + seq + 1) - t0;
+  const int keep = __ldg(sig_keep + seg);
+  float* out = theta + (size_t)seg * s.Hq + h;
+  if (keep <= 0 || keep >= L) {
+    if (threadIdx.x == 0) *out = keep <= 0 ? __int_as_float(0x7F800000) : __int_as_float(0xFF800000);
+    return;
+  }
+  const float* row = scores + ((size_t)layer * s.Hq + h) * s.T + t0;
+  const int lane = threadIdx.x & 31;
+
+  uint32_t prefix = 0;       // selected high digits so far
+  uint32_t k_rem = keep;     // rank among the elements that share the prefix
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = threadIdx.x; i < 256; i += kSelectThreads) hist[i] = 0;
+    __syncthreads();
+    const uint32_t hi_mask = shift == 24 ? 0u : (0xFFFFFFFFu << (shift + 8));
+    for (int base = 0; base < L; base += kSelectThreads) {
+      const int i = base + threadIdx.x;
+      const bool in = i < L;
+      const uint32_t key = in ? order_key(__ldg(row + i)) : 0u;
+      const bool live = in && ((key & hi_mask) == prefix);
+      const uint32_t digit = (key >> shift) & 0xFFu;
+      const unsigned voters = __ballot_sync(0xFFFFFFFFu, live);
+      if (live) {
+        const unsigned peers = __match_any_sync(voters, digit);
+        if ((peers & ((1u << lane) - 1u)) == 0) atomicAdd(&hist[digit], __popc(peers));
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      // lane l owns the 8 bins 255-8l .. 248-8l (descending order of value)
+      uint32_t local = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) local += hist[255 - 8 * lane - j];
+      uint32_t incl = local;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += v;
+      }
+      const uint32_t excl = incl - local;
+      if (excl < k_rem && k_rem <= incl) {
+        uint32_t acc = excl;
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t c = hist[255 - 8 * lane - j];
+          if (k_rem <= acc + c) {
+            sel_prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
+            sel_k = k_rem - acc;
+            break;
+          }
+          acc += c;
+        }
+      }
+    }
+    __syncthreads();
+    prefix = sel_prefix;
+    k_rem = sel_k;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = key_to_float(prefix);
+}
+
+__global__ void __launch_bounds__(256)
+binarise_pack_kernel(Shape s, const float* __restrict__ scores, const float* __restrict__ theta,
+                     uint32_t* __restrict__ sigs) {
+  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= (long long)s.n_layers * s.T) return;
+  const int layer = (int)(gid / s.T), tok = (int)(gid - (long long)layer * s.T);
+  const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
+  const float* sc = scores + (size_t)layer * s.Hq * s.T + tok;
+  const float* th = theta + ((size_t)layer * s.n_seqs + seq) * s.Hq;
+  uint32_t* out = sigs + ((size_t)layer * s.T + tok) * s.W;
+  for (int w = 0; w < s.W; ++w) {
+    uint32_t word = 0;
+    const int h_end = min(32, s.Hq - 32 * w);
+    for (int b = 0; b < h_end; ++b) {
+      const int h = 32 * w + b;
+      word |= (uint32_t)(__ldg(sc + (size_t)h * s.T) >= __ldg(th + h)) << b;
+    }
+    out[w] = word;
+  }
+}
+
+}  // namespace
+
+int launch_signature(const Shape& s, const float* scores, const int32_t* sig_keep, const float* theta_in,
+                     uint32_t* sigs, float* theta, cudaStream_t stream) {
+  if (s.T == 0) return KVCRUSH_OK;
+  const float* th = theta_in;
+  if (!theta_in) {
+    const unsigned blocks = (unsigned)s.n_layers * s.n_seqs * s.Hq;
+    theta_select_kernel<<<blocks, kSelectThreads, 0, stream>>>(s, scores, sig_keep, theta);
+    if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+    th = theta;
+  }
+  const long long n = (long long)s.n_layers * s.T;
+  binarise_pack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, scores, th, sigs);
+  return check_launch();
+}
+
+}  // namespace kvc

@@ -132,7 +132,12 @@ def to_storage(x: np.ndarray, dtype: str) -> np.ndarray:
     bf16 -> uint16 bit patterns, fp16 -> numpy float16, fp32 -> float32.
     """
     if dtype == BF16:
-        return f32_to_bf16_bits(x)
+        try:                                     # same rounding, multi-threaded
+            import torch
+            t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.bfloat16)
+            return t.view(torch.int16).numpy().view(np.uint16)
+        except ImportError:
+            return f32_to_bf16_bits(x)
     if dtype == FP16:
         return x.astype(np.float16)
     if dtype == FP32:
