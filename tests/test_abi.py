@@ -1,0 +1,100 @@
+"""The C-ABI library: it loads, exports every symbol the header declares, and rejects bad
+arguments on the host before anything is launched (none of these calls touches a GPU)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2503_00022_b200 import binding as B
+from paper_2503_00022_b200 import build as kbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    kbuild.build()
+    return B.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "kvcrush.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(kvcrush_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = _declared()
+    assert set(B.EXPORTS) <= set(names) and len(names) >= 7
+    for n in names:
+        assert hasattr(lib, n), n
+    assert B.kvcrush_version() >= 100
+    assert B.strerror(B.ERR_WORKSPACE) == "workspace missing or too small"
+    assert B.strerror(0) == "ok"
+
+
+def _problem(**over):
+    cu = np.asarray(over.pop("cu", [0, 100]), dtype=np.int32)
+    kw = dict(n_layers=1, n_seqs=len(cu) - 1, n_q_heads=8, n_kv_heads=4, head_dim=64, total_tokens=int(cu[-1]),
+              max_seqlen=int(np.diff(cu).max()), causal=1, softmax_scale=0.0, reserved=0,
+              cu_seqlens_host=cu.ctypes.data, cu_seqlens_dev=0x1000)
+    kw.update(over)
+    p = B.ProblemStruct(**kw)
+    p._keep = cu
+    return p
+
+
+def test_workspace_sizes_and_shape_validation(lib):
+    out = ctypes.c_size_t(0)
+    p = _problem()
+    assert lib.kvcrush_workspace_size(ctypes.byref(p), B.STAGE_SCORE, ctypes.byref(out)) == 0
+    assert out.value >= 8 * 100 * 4 and out.value % 256 == 0
+    assert lib.kvcrush_workspace_size(ctypes.byref(p), B.STAGE_SELECT, ctypes.byref(out)) == 0
+    assert out.value >= 100 * 12
+    assert lib.kvcrush_workspace_size(ctypes.byref(p), B.STAGE_COMPACT, ctypes.byref(out)) == 0 and out.value == 0
+    assert lib.kvcrush_workspace_size(ctypes.byref(p), 9, ctypes.byref(out)) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_workspace_size(None, 0, ctypes.byref(out)) == B.ERR_INVALID_ARG
+    for bad in (dict(n_kv_heads=3), dict(n_layers=0), dict(total_tokens=99), dict(max_seqlen=50),
+                dict(cu_seqlens_dev=None), dict(cu=[0, 60, 40])):
+        q = _problem(**bad)
+        assert lib.kvcrush_workspace_size(ctypes.byref(q), 0, ctypes.byref(out)) == B.ERR_INVALID_ARG, bad
+    assert lib.kvcrush_workspace_size(ctypes.byref(_problem(n_q_heads=256, n_kv_heads=256)), 0,
+                                      ctypes.byref(out)) == B.ERR_UNSUPPORTED
+
+
+def test_entry_points_reject_bad_arguments_before_launch(lib):
+    p = _problem()
+    t = B.TensorStruct(0x10000, B.BF16, 0, 100 * 8 * 64, 8 * 64, 64)
+    odd = B.TensorStruct(0x10002, B.BF16, 0, 100 * 8 * 64, 8 * 64, 64)
+    f16 = B.TensorStruct(0x10000, B.FP16, 0, 100 * 8 * 64, 8 * 64, 64)
+    r = ctypes.byref
+    # score: NULL outputs, misaligned tensor, dtype mismatch / unsupported, missing workspace
+    assert lib.kvcrush_score(r(p), r(t), r(t), None, None, None, 0, 0, None, 0, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_score(r(p), r(odd), r(t), None, 0x100, None, 0, 0, 0x100, 1 << 20, 0x100, None) == B.ERR_MISALIGNED
+    assert lib.kvcrush_score(r(p), r(f16), r(f16), None, 0x100, None, 0, 0, 0x100, 1 << 20, 0x100, None) == B.ERR_UNSUPPORTED
+    assert lib.kvcrush_score(r(p), r(t), r(f16), None, 0x100, None, 0, 0, 0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_score(r(p), r(t), r(t), None, 0x100, None, 0, 0, None, 0, 0x100, None) == B.ERR_WORKSPACE
+    assert lib.kvcrush_score(r(p), r(t), r(t), None, 0x100, None, 0, 7, 0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
+    # signature: needs a rank or explicit thresholds; needs workspace when theta_out is NULL
+    assert lib.kvcrush_signature(r(p), 0x100, None, None, 0x100, None, None, 0, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_signature(r(p), 0x100, 0x100, None, 0x100, None, None, 0, 0x100, None) == B.ERR_WORKSPACE
+    # select: anchor mode range, explicit anchor needs bits, workspace
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 5, None, 0, 0x100, 0x100, None, 0x100, 1 << 20,
+                              0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, B.ANCHOR_EXPLICIT, None, 0, 0x100, 0x100, None,
+                              0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, 0x100, 0x100, None, 0x100, 16,
+                              0x100, None) == B.ERR_WORKSPACE
+    # compact: V without V_out, dtype mismatch, negative count
+    assert lib.kvcrush_compact(r(p), r(t), r(t), 0x100, 0x100, 10, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_compact(r(p), r(t), None, 0x100, 0x100, 10, r(f16), None, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_compact(r(p), r(t), None, 0x100, 0x100, -1, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        B.lib()
