@@ -201,3 +201,48 @@ SIMT_CASES = [
 @pytest.mark.parametrize("w", SIMT_CASES, ids=lambda w: w.name)
 def test_score_simt_matches_oracle(B, w):
     _score_case(B, w, B.SCORE_SIMT)
+
+
+TENSOR_CASES = [
+    inputs.Workload("tc_one_tile", 1, 2, 2, 128, (128,), inputs.BF16, inputs.BF16, 0.25, base_seed=31),
+    inputs.Workload("tc_ragged_tail", 1, 4, 4, 128, (700,), inputs.BF16, inputs.BF16, 0.25, base_seed=32),
+    inputs.Workload("tc_gqa_varlen", 2, 8, 2, 128, (300, 1, 129, 1000), inputs.BF16, inputs.BF16, 0.25, base_seed=33),
+    inputs.Workload("tc_d64", 1, 4, 2, 64, (513, 64), inputs.BF16, inputs.BF16, 0.25, base_seed=34),
+    inputs.Workload("tc_noncausal", 1, 4, 4, 128, (333, 260), inputs.BF16, inputs.BF16, 0.25, base_seed=35, causal=False),
+    inputs.Workload("tc_2k", 1, 8, 8, 128, (2048,), inputs.BF16, inputs.BF16, 0.25, base_seed=36),
+]
+
+
+@pytest.mark.parametrize("w", TENSOR_CASES, ids=lambda w: w.name)
+def test_score_tensor_matches_oracle(B, w):
+    g = _score_case(B, w, B.SCORE_TENSOR)
+    # the CUDA-core kernels see the same inputs: the two device paths agree far inside the tolerance
+    import torch
+    dev = _dev()
+    lis, q, k, _, _ = TL.stack_layers(w, range(w.n_layers), with_cache=False)
+    prob = B.Problem(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, causal=w.causal, device=dev)
+    scores = torch.empty((w.n_layers, w.n_q_heads, w.total_tokens), dtype=torch.float32, device=dev)
+    ws = torch.empty(B.kvcrush_workspace_size(prob, B.STAGE_SCORE), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    B.kvcrush_score(prob, TL.torch_storage(q, w.qk_dtype, dev), TL.torch_storage(k, w.qk_dtype, dev), scores,
+                    impl=B.SCORE_SIMT, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(g, scores.cpu().numpy(), rtol=2e-4, atol=1e-6)
+
+
+def test_score_tensor_rejects_fp32_and_auto_falls_back_to_cuda_cores(B):
+    import torch
+    dev = _dev()
+    w = SIMT_CASES[0]
+    lis, q, k, _, _ = TL.stack_layers(w, range(1), with_cache=False)
+    prob = B.Problem(1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, device=dev)
+    dq, dk = TL.torch_storage(q, w.qk_dtype, dev), TL.torch_storage(k, w.qk_dtype, dev)
+    scores = torch.empty((1, w.n_q_heads, w.total_tokens), dtype=torch.float32, device=dev)
+    ws = torch.empty(B.kvcrush_workspace_size(prob, B.STAGE_SCORE), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    with pytest.raises(B.KvcrushError) as e:
+        B.kvcrush_score(prob, dq, dk, scores, impl=B.SCORE_TENSOR, workspace=ws, status=status)
+    assert e.value.code == B.ERR_UNSUPPORTED
+    B.kvcrush_score(prob, dq, dk, scores, impl=B.SCORE_AUTO, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert torch.isfinite(scores).all()
