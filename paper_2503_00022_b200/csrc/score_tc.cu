@@ -206,8 +206,8 @@ struct Aux {                         // lives at kAuxOff
   uint32_t tmem_base;
   int abort_flag;
   int item[4];                       // seq, tile, n_tiles
-  float lse_sh[2][2][kTile];         // [group][buffer][query in tile]   (sweep 2)
-  float part[2][kTile];              // group 1 partials handed to group 0
+  alignas(16) float lse_sh[2][2][kTile];         // [group][buffer][query in tile]   (sweep 2)
+  alignas(16) float part[2][kTile];              // group 1 partials handed to group 0
 };
 
 template <int D, bool kColsum>
