@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the KVCrush compression pass (score -> signature -> select -> compact).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one batch of synthetic input (every layer of
+the workload).  Prints ONE JSON line.  `value` is prompt tokens compressed per second with
+the inputs resident in HBM; `e2e` is the same through host buffers (pinned host -> device
+copies of Q, K and the K/V cache, device -> host copy of the kept indices and the reduced
+cache inside the timed region).  `roofline` covers the dominant kernel (the tensor-core score
+sweeps); `cpu_baseline` is the float64 oracle timed on this machine's host cores on a bounded
+sample.  With N > 1 (torchrun) every rank runs its own replica of the workload: the pass has
+no exchange step, so there is no collective on the data path (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_00022_b200 import inputs  # noqa: E402
+
+METRIC = "prompt tokens compressed/s (score+select+compact)"
+UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "cfg3_llama2_32l_8k"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ---------------------------------------------------------------------------------------------
+# workload arithmetic (algorithmic work, independent of how the kernels do it)
+# ---------------------------------------------------------------------------------------------
+
+def algorithmic_work(w: inputs.Workload):
+    """Per step (all layers).  Causal entries per head = L(L+1)/2; 2*D flops each; two sweeps."""
+    entries = sum(L * (L + 1) // 2 if w.causal else L * L for L in w.seqlens)
+    flops_per_sweep = 2 * w.head_dim * entries * w.n_q_heads * w.n_layers
+    b_imp, b_rep = w.budgets()
+    kept = int((b_imp + b_rep).sum())
+    eb = inputs.storage_itemsize(w.cache_dtype)
+    compact_bytes = 2 * 2 * kept * w.n_kv_heads * w.head_dim * eb * w.n_layers        # K and V, read + write
+    T, W = w.total_tokens, (w.n_q_heads + 31) // 32
+    signature_bytes = (4 * w.n_q_heads + 4 * W) * T * w.n_layers
+    select_bytes = (4 * w.n_q_heads + 4 * W) * T * w.n_layers + 4 * kept * w.n_layers
+    return dict(score_flops=2 * flops_per_sweep, exps=2 * entries * w.n_q_heads * w.n_layers,
+                compact_bytes=compact_bytes, signature_bytes=signature_bytes, select_bytes=select_bytes, kept=kept)
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t_begin: float, t_end: float):
+        if self.proc is None:
+            return None
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t_begin <= t <= t_end + 0.2] or [r for _, r in self.rows]
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return None
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+
+
+# ---------------------------------------------------------------------------------------------
+# input staging
+# ---------------------------------------------------------------------------------------------
+
+def host_inputs(w: inputs.Workload, pinned: bool):
+    """All layers of the workload as host torch tensors (storage dtypes), drawn in parallel."""
+    import torch
+    tq = {inputs.BF16: torch.bfloat16, inputs.FP32: torch.float32}[w.qk_dtype]
+    tc = {inputs.BF16: torch.bfloat16, inputs.FP16: torch.float16, inputs.FP32: torch.float32}[w.cache_dtype]
+    T = w.total_tokens
+    mk = dict(pin_memory=pinned)
+    q = torch.empty((w.n_layers, T, w.n_q_heads, w.head_dim), dtype=tq, **mk)
+    k = torch.empty((w.n_layers, T, w.n_kv_heads, w.head_dim), dtype=tq, **mk)
+    kc = k if w.cache_dtype == w.qk_dtype else torch.empty((w.n_layers, T, w.n_kv_heads, w.head_dim), dtype=tc, **mk)
+    vc = torch.empty((w.n_layers, T, w.n_kv_heads, w.head_dim), dtype=tc, **mk)
+
+    def as_t(a, dt):
+        t = torch.from_numpy(a.view(np.int16)) if dt == inputs.BF16 else torch.from_numpy(a)
+        return t.view(torch.bfloat16) if dt == inputs.BF16 else t
+
+    def one(layer):
+        li = inputs.layer_inputs(w, layer)
+        q[layer].copy_(as_t(li.q, w.qk_dtype))
+        k[layer].copy_(as_t(li.k, w.qk_dtype))
+        if kc is not k:
+            kc[layer].copy_(as_t(li.k_cache, w.cache_dtype))
+        vc[layer].copy_(as_t(li.v_cache, w.cache_dtype))
+
+    with ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 8)) as ex:
+        list(ex.map(one, range(w.n_layers)))
+    return q, k, kc, vc
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------------------------
+
+def oracle_sample(w: inputs.Workload, max_heads=None):
+    """Times the float64 oracle on a bounded sample of the workload and scales to one step.
+
+    Sample: the score step for the first H_s query heads of layer 0 (H_s = host threads, at most
+    all heads) on the longest sequence, and signature + selection + compaction of layer 0's longest
+    sequence on seeded stand-in scores.  The step estimate scales the score time by
+    (layers * heads * causal entries) / sampled entries and the rest by layers * sequences-length share.
+    """
+    from oracle import kvcrush_oracle as O
+    threads = O.n_threads()
+    s_long = int(np.argmax(w.seqlens))
+    L = w.seqlens[s_long]
+    cu = w.cu_seqlens
+    li = inputs.layer_inputs(w, 0)
+    hs = min(w.n_q_heads, max(1, threads if max_heads is None else max_heads))
+    G = w.n_q_heads // w.n_kv_heads
+    hk = sorted(set(h // G for h in range(hs)))
+    a, b = int(cu[s_long]), int(cu[s_long + 1])
+    q = inputs.widen(li.q[a:b, :hs], w.qk_dtype)
+    # keep the GQA mapping of the sampled heads: expand their KV heads to one per query head
+    k = inputs.widen(li.k[a:b][:, [h // G for h in range(hs)]], w.qk_dtype)
+    del hk
+    t0 = time.perf_counter()
+    O.scores(q, k, w.causal)
+    t_score = time.perf_counter() - t0
+    entries_sample = hs * (L * (L + 1) // 2 if w.causal else L * L)
+    entries_step = w.n_layers * w.n_q_heads * sum(x * (x + 1) // 2 if w.causal else x * x for x in w.seqlens)
+    b_imp, b_rep = w.budgets()
+    s32 = inputs.random_scores(w.n_q_heads, L, 7)
+    t0 = time.perf_counter()
+    theta = O.thresholds(s32, int(b_imp[s_long] + b_rep[s_long]))
+    sig = O.signatures(s32, theta)
+    idx, _ = O.select(s32, sig, int(b_imp[s_long]), int(b_rep[s_long]), w.n_kv_heads)
+    O.compact(li.k_cache[a:b], idx)
+    O.compact(li.v_cache[a:b], idx)
+    t_rest = time.perf_counter() - t0
+    step_s = t_score * entries_step / entries_sample + t_rest * w.n_layers * w.total_tokens / L
+    desc = (f"score: layer 0, {hs} of {w.n_q_heads} heads, L={L} ({t_score:.2f} s); signature+select+compact: "
+            f"layer 0, L={L} on seeded stand-in scores ({t_rest:.2f} s); scaled to {w.n_layers} layers x "
+            f"{w.n_q_heads} heads x {w.total_tokens} tokens")
+    return dict(value=w.total_tokens / step_s, unit=UNIT, cores=threads, kind="oracle", sample=desc,
+                est_step_s=step_s)
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import kvcrush_oracle as O
+    O.build_c()
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample(w, max_heads=2)
+    vals = [oracle_sample(w) for _ in range(max(1, min(args.steps, 3)))]
+    best = max(vals, key=lambda v: v["value"])
+    value = float(np.mean([v["value"] for v in vals]))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * w.total_tokens / value, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
+                   "head_dim": w.head_dim, "seqlens": list(w.seqlens)[:4], "note": "each step is a bounded sample scaled to the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": best["cores"], "kind": "oracle", "sample": best["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2503_00022_b200 import binding as B
+    from paper_2503_00022_b200 import build as kbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        kbuild.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    hq, hk, hkc, hvc = host_inputs(w, pinned=True)
+    q, k = hq.to(dev, non_blocking=True), hk.to(dev, non_blocking=True)
+    kc = k if hkc is hk else hkc.to(dev, non_blocking=True)
+    vc = hvc.to(dev, non_blocking=True)
+    tc = vc.dtype
+    prob = B.Problem(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, causal=w.causal, device=dev)
+    b_imp, b_rep = w.budgets()
+    cp = B.CompressionPass(prob, b_imp[None, :], b_rep[None, :], cache_dtype=tc, impl=B.SCORE_AUTO)
+    torch.cuda.synchronize()
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+
+    def step(marks=None):
+        if marks: marks[0].record()
+        cp.score(q, k)
+        if marks: marks[1].record()
+        cp.signature()
+        if marks: marks[2].record()
+        cp.select()
+        if marks: marks[3].record()
+        cp.compact(kc, vc)
+        if marks: marks[4].record()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    cp.check_status()
+    sampler = ClockSampler(local) if rank == 0 else None
+    t_begin = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        step(ev[i])
+    e1.record()
+    barrier()
+    t_end = time.time()
+    clocks = sampler.stop(t_begin, t_end) if sampler else None
+    cp.check_status()
+    total_ms = e0.elapsed_time(e1)
+    stage_ms = np.asarray([[ev[i][j].elapsed_time(ev[i][j + 1]) for j in range(4)] for i in range(args.steps)]).mean(axis=0)
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+
+    # ---- end to end through host buffers: H2D of the step's inputs, D2H of the kept set and reduced cache ----
+    e2e_steps = max(1, min(args.steps, 3))
+    h_idx = torch.empty(cp.idx.shape, dtype=cp.idx.dtype, pin_memory=True)
+    h_ko = torch.empty(cp.k_out.shape, dtype=cp.k_out.dtype, pin_memory=True)
+    h_vo = torch.empty(cp.v_out.shape, dtype=cp.v_out.dtype, pin_memory=True)
+
+    def e2e_step():
+        q.copy_(hq, non_blocking=True)
+        k.copy_(hk, non_blocking=True)
+        if kc is not k:
+            kc.copy_(hkc, non_blocking=True)
+        vc.copy_(hvc, non_blocking=True)
+        step()
+        h_idx.copy_(cp.idx, non_blocking=True)
+        h_ko.copy_(cp.k_out, non_blocking=True)
+        h_vo.copy_(cp.v_out, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_ms /= e2e_steps
+    nbytes = lambda t: t.numel() * t.element_size()  # noqa: E731
+    h2d = nbytes(hq) + nbytes(hk) + (nbytes(hkc) if hkc is not hk else 0) + nbytes(hvc)
+    d2h = nbytes(h_idx) + nbytes(h_ko) + nbytes(h_vo)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    work = algorithmic_work(w)
+    score_s = stage_ms[0] * 1e-3
+    tensor_path = B.lib() is not None and w.qk_dtype == inputs.BF16 and w.head_dim in (64, 128)
+    achieved_tf = work["score_flops"] / score_s / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"]
+    traffic = None
+    roofline = {"bound": "tensor" if tensor_path else "alu", "kernel": "score_tc_kernel (two sweeps per step)" if tensor_path else "score SIMT",
+                "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
+                "traffic": traffic, "peak_source": peaks["source"] + " (sustained bf16)",
+                "frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved_tf / 2250.0,
+                "exps_per_s": work["exps"] / score_s}
+    hbm = peaks["hbm_gbs"]
+    stages = {
+        "score_ms": float(stage_ms[0]), "signature_ms": float(stage_ms[1]), "select_ms": float(stage_ms[2]),
+        "compact_ms": float(stage_ms[3]),
+        "compact_gbs": work["compact_bytes"] / (stage_ms[3] * 1e-3) / 1e9,
+        "compact_frac_hbm": work["compact_bytes"] / (stage_ms[3] * 1e-3) / 1e9 / hbm,
+        "signature_gbs": work["signature_bytes"] / (stage_ms[1] * 1e-3) / 1e9,
+        "select_gbs": work["select_bytes"] / (stage_ms[2] * 1e-3) / 1e9,
+        "hbm_peak_gbs": hbm, "hbm_peak_source": peaks["source"],
+    }
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import kvcrush_oracle as O
+        O.build_c()
+        cpu = oracle_sample(w)
+        cpu.pop("est_step_s", None)
+
+    tokens = w.total_tokens * world
+    line = {
+        "metric": METRIC, "value": tokens / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w.qk_dtype == inputs.BF16 else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
+                   "head_dim": w.head_dim, "n_seqs": w.n_seqs, "total_tokens": w.total_tokens,
+                   "budget_per_seq": [int(b_imp[0] + b_rep[0])], "cache_dtype": w.cache_dtype,
+                   "l2": "inputs larger than L2 (%.1f GiB resident per step)" % (h2d / 2 ** 30),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "layer_tokens_per_s": tokens * w.n_layers / (ms_per_step * 1e-3),
+        "roofline": roofline, "stages": stages, "cpu_baseline": cpu,
+        "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": e2e_ms},
+        "gpu_launches": 7 * args.steps,
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--layers", type=int, default=0, help="run only this many layers of the workload (profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = inputs.paper_workloads()[args.workload]
+    if args.layers:
+        w = inputs.shrink(w, args.layers)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
