@@ -51,6 +51,7 @@ extern "C" {
 #define KVCRUSH_ERR_MISALIGNED    (-3)   /* pointer or stride breaks an alignment rule       */
 #define KVCRUSH_ERR_WORKSPACE     (-4)   /* workspace NULL or too small                      */
 #define KVCRUSH_ERR_CUDA          (-5)   /* a CUDA runtime / driver call failed              */
+#define KVCRUSH_ERR_STATIC_LIMIT  (-6)   /* problem larger than a built-in scratch array     */
 
 /* status_dev[0] values */
 #define KVCRUSH_DEV_OK             0
@@ -189,6 +190,33 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
                     const int32_t* cu_kept_dev, const int32_t* idx_dev, int64_t total_kept,
                     const kvcrush_tensor_t* K_out, const kvcrush_tensor_t* V_out,
                     int32_t* status_dev, void* stream);
+
+/*
+ * Stage 2 without caller-provided scratch (the paper has no counterpart; this is a packaging
+ * variant of kvcrush_signature for hosts that cannot hand over device memory).
+ *
+ * Who needs it: code that runs where device allocation is off the table - a plug-in inside a
+ * serving engine that owns the whole memory pool and forbids cudaMalloc in its hot path, a
+ * callback that must not trigger the implicit device synchronisation an allocation causes, or an
+ * embedding that simply has no allocator to offer for the thresholds' scratch.
+ *
+ * Same computation and outputs as kvcrush_signature with sig_keep_dev (no explicit thresholds,
+ * no theta output): the per-head thresholds live in a scratch array that is part of the library
+ * image (file-scope __device__ memory, KVCRUSH_STATIC_THETA_MAX floats = 256 KiB, resident on every
+ * GPU that loads the library until the process exits).  The call allocates nothing and frees nothing.
+ *   - n_layers * n_seqs * n_q_heads must not exceed KVCRUSH_STATIC_THETA_MAX, otherwise
+ *     KVCRUSH_ERR_STATIC_LIMIT is returned and nothing runs.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress with that device current); make that first call outside any stream
+ *     capture.  Later calls reuse the address.
+ *   - All calls share the one array per device and it keeps whatever the previous call left.  Nothing
+ *     in it has to start at zero: every threshold a call reads is written earlier in that same call.
+ *     Two calls that overlap on the GPU (different streams, no ordering) race on it; serialise them.
+ */
+#define KVCRUSH_STATIC_THETA_MAX 65536
+int kvcrush_signature_static(const kvcrush_problem_t* problem, const float* scores_dev,
+                             const int32_t* sig_keep_dev, uint32_t* sigs_dev,
+                             int32_t* status_dev, void* stream);
 
 /* Text for a return code. */
 const char* kvcrush_strerror(int code);

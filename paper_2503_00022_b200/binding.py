@@ -18,6 +18,8 @@ LIB_PATH = os.path.join(_PKG, "libkvcrush.so")
 
 # constants of include/kvcrush.h
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_WORKSPACE, ERR_CUDA = 0, -1, -2, -3, -4, -5
+ERR_STATIC_LIMIT = -6
+STATIC_THETA_MAX = 65536
 DEV_OK, DEV_TIMEOUT = 0, 1
 BF16, FP16, FP32 = 0, 1, 2
 STAGE_SCORE, STAGE_SIGNATURE, STAGE_SELECT, STAGE_COMPACT = 0, 1, 2, 3
@@ -25,7 +27,7 @@ ANCHOR_ALTERNATE, ANCHOR_MEAN, ANCHOR_EXPLICIT = 0, 1, 2
 SCORE_AUTO, SCORE_SIMT, SCORE_TENSOR = 0, 1, 2
 
 EXPORTS = ("kvcrush_workspace_size", "kvcrush_score", "kvcrush_signature", "kvcrush_select",
-           "kvcrush_compact", "kvcrush_strerror", "kvcrush_version")
+           "kvcrush_compact", "kvcrush_strerror", "kvcrush_version", "kvcrush_signature_static")
 
 
 class ProblemStruct(ctypes.Structure):
@@ -68,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.kvcrush_signature.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_compact.argtypes = [P, T, T, vp, vp, i64, T, T, vp, vp]
+        L.kvcrush_signature_static.argtypes = [P, vp, vp, vp, vp, vp]
         L.kvcrush_strerror.argtypes = [i32]
         L.kvcrush_strerror.restype = ctypes.c_char_p
         L.kvcrush_version.argtypes = []
@@ -157,6 +160,15 @@ def kvcrush_signature(problem: Problem, scores, sigs, *, sig_keep=None, theta_in
     _check(lib().kvcrush_signature(problem.ref, _ptr(scores), _ptr(sig_keep), _ptr(theta_in), _ptr(sigs),
                                    _ptr(theta_out), _ptr(workspace), ws_bytes, _ptr(status),
                                    _stream() if stream is None else stream), "kvcrush_signature")
+
+
+def kvcrush_signature_static(problem: Problem, scores, sigs, sig_keep, *, status=None,
+                             stream: Optional[int] = None) -> None:
+    """kvcrush_signature without a workspace: the thresholds' scratch is device memory built into the
+    library (at most STATIC_THETA_MAX thresholds).  For hosts that must not allocate; calls on one
+    device must not overlap."""
+    _check(lib().kvcrush_signature_static(problem.ref, _ptr(scores), _ptr(sig_keep), _ptr(sigs), _ptr(status),
+                                          _stream() if stream is None else stream), "kvcrush_signature_static")
 
 
 def kvcrush_select(problem: Problem, scores, sigs, budget_imp, budget_rep, cu_kept, idx, *, kind=None,

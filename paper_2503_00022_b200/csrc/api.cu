@@ -51,6 +51,10 @@ size_t signature_ws(const Shape& s) { return round_up((size_t)s.n_layers * s.n_s
 
 }  // namespace
 
+namespace kvc {
+int shape_from_problem(const kvcrush_problem_t* problem, Shape* out) { return make_shape(problem, out); }
+}  // namespace kvc
+
 extern "C" {
 
 int kvcrush_workspace_size(const kvcrush_problem_t* problem, int stage, size_t* bytes) {
@@ -174,6 +178,7 @@ const char* kvcrush_strerror(int code) {
     case KVCRUSH_ERR_MISALIGNED: return "misaligned pointer or stride";
     case KVCRUSH_ERR_WORKSPACE: return "workspace missing or too small";
     case KVCRUSH_ERR_CUDA: return "CUDA call failed";
+    case KVCRUSH_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch array";
     default: return "unknown error";
   }
 }

@@ -69,6 +69,9 @@ int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, con
                    const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,
                    cudaStream_t stream);
 
+// Validates a problem description and fills the device-side view (defined in api.cu).
+int shape_from_problem(const kvcrush_problem_t* problem, Shape* out);
+
 inline int check_launch() { return cudaGetLastError() == cudaSuccess ? KVCRUSH_OK : KVCRUSH_ERR_CUDA; }
 
 }  // namespace kvc

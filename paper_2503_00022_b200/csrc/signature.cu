@@ -133,4 +133,47 @@ int launch_signature(const Shape& s, const float* scores, const int32_t* sig_kee
   return check_launch();
 }
 
+// ---------------------------------------------------------------------------------------------------
+// kvcrush_signature_static: the same two kernels, thresholds kept in library-owned device memory.
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+// Thresholds of one call, [n_layers][n_seqs][n_q_heads].  Lives in the library image on every device.
+static __device__ __align__(256) float g_static_theta[KVCRUSH_STATIC_THETA_MAX];
+
+constexpr int kMaxDevices = 64;
+
+// Device address of g_static_theta on the current device.  In host code the symbol's name is only a
+// handle; the address a kernel can use comes from cudaGetSymbolAddress, looked up once per device.
+int static_theta_ptr(float** out) {
+  static float* cached[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return KVCRUSH_ERR_CUDA;
+  float* p = __atomic_load_n(&cached[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_static_theta) != cudaSuccess || !addr) return KVCRUSH_ERR_CUDA;
+    p = static_cast<float*>(addr);
+    __atomic_store_n(&cached[dev], p, __ATOMIC_RELEASE);
+  }
+  *out = p;
+  return KVCRUSH_OK;
+}
+
+}  // namespace
 }  // namespace kvc
+
+extern "C" int kvcrush_signature_static(const kvcrush_problem_t* problem, const float* scores_dev,
+                                        const int32_t* sig_keep_dev, uint32_t* sigs_dev,
+                                        int32_t* status_dev, void* stream) {
+  kvc::Shape s;
+  const int rc = kvc::shape_from_problem(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if (!scores_dev || !sig_keep_dev || !sigs_dev || !status_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if ((long long)s.n_layers * s.n_seqs * s.Hq > KVCRUSH_STATIC_THETA_MAX) return KVCRUSH_ERR_STATIC_LIMIT;
+  float* theta = nullptr;
+  const int prc = kvc::static_theta_ptr(&theta);
+  if (prc != KVCRUSH_OK) return prc;
+  return kvc::launch_signature(s, scores_dev, sig_keep_dev, nullptr, sigs_dev, theta,
+                               static_cast<cudaStream_t>(stream));
+}
