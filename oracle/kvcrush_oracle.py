@@ -84,7 +84,7 @@ def _c_lib():
         lib.kvcrush_oracle_scores.restype = ctypes.c_int
         lib.kvcrush_oracle_scores.argtypes = [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
-            ctypes.c_int, ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p]
+            ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
         lib.kvcrush_oracle_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -95,11 +95,13 @@ def n_threads() -> int:
 
 
 def scores(q: np.ndarray, k: np.ndarray, causal: bool = True, scale: Optional[float] = None,
-           normalize: bool = False) -> Tuple[np.ndarray, np.ndarray]:
+           normalize: bool = False, rows: Optional[Tuple[int, int]] = None) -> Tuple[np.ndarray, np.ndarray]:
     """Column sums of the softmax attention matrix, one sequence (Algorithm 1).
 
     q [L, Hq, D], k [L, Hkv, D] float64.  Returns (c [Hq, L], lse [Hq, L]) float64;
     with ``normalize`` the first is w = c / L.  Runs the C routine (row by row).
+    ``rows=(j0, j1)`` visits only the queries j0 <= j < j1: c is then the sum over those rows
+    (the complete column sum for keys t >= j0 when causal) and lse is valid on those rows only.
     """
     q = np.ascontiguousarray(q, dtype=np.float64)
     k = np.ascontiguousarray(k, dtype=np.float64)
@@ -110,8 +112,9 @@ def scores(q: np.ndarray, k: np.ndarray, causal: bool = True, scale: Optional[fl
         scale = 1.0 / np.sqrt(D)
     c = np.zeros((Hq, L), dtype=np.float64)
     lse = np.zeros((Hq, L), dtype=np.float64)
+    j0, j1 = (0, L) if rows is None else (int(rows[0]), int(rows[1]))
     rc = _c_lib().kvcrush_oracle_scores(q.ctypes.data, k.ctypes.data, L, Hq, Hkv, D, int(bool(causal)),
-                                        float(scale), c.ctypes.data, lse.ctypes.data)
+                                        float(scale), j0, j1, c.ctypes.data, lse.ctypes.data)
     if rc != 0:
         raise RuntimeError("kvcrush_oracle_scores failed")
     if normalize and L > 0:

@@ -29,12 +29,17 @@
  * causal != 0: query j attends keys t <= j; otherwise all keys
  * colsum [Hq][L] out: c_h(t)
  * lse    [Hq][L] out (may be NULL): log sum_t exp(s(j,t)) for every query j
+ * j_begin, j_end: only the query rows j_begin <= j < j_end are visited (0, L = all of them).
+ *        With a partial range colsum holds the sum over those rows only - which is the complete
+ *        c_h(t) for every key t >= j_begin of a causal sequence (earlier queries do not see t) -
+ *        and lse is written for those rows only.  Used to check samples of long sequences.
  * returns 0, or -1 on bad arguments / allocation failure
  */
 int kvcrush_oracle_scores(const double *Q, const double *K, int L, int Hq, int Hkv, int D,
-                          int causal, double scale, double *colsum, double *lse)
+                          int causal, double scale, int j_begin, int j_end, double *colsum, double *lse)
 {
     if (L < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return -1;
+    if (j_begin < 0 || j_end > L || j_begin > j_end) return -1;
     const int G = Hq / Hkv;
     int failed = 0;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -48,7 +53,7 @@ int kvcrush_oracle_scores(const double *Q, const double *K, int L, int Hq, int H
             continue;
         }
         const int hk = h / G;
-        for (int j = 0; j < L; ++j) {
+        for (int j = j_begin; j < j_end; ++j) {
             const double *q = Q + ((size_t)j * Hq + h) * D;
             const int n = causal ? j + 1 : L;
             double m = -INFINITY;

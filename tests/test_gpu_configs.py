@@ -1,0 +1,247 @@
+"""GPU parity on the five benchmark shapes, through the C ABI, in the launch configuration bench.py
+times (all layers in one call per stage).
+
+Small shapes (1, 2) are compared with the oracle element by element, end to end.  For the large
+shapes the oracle computes what it can in seconds - all heads of one layer, a few heads of other
+layers, the complete tail columns and sampled rows of very long sequences - and everything else is
+checked through properties that hold at any size: column sums of a head total the number of
+queries, kept counts equal the budget, kept lists are strictly ascending, and the oracle's
+selection run on the GPU's own float32 scores reproduces the GPU's kept set bit for bit."""
+import numpy as np
+import pytest
+
+from oracle import kvcrush_oracle as O
+from paper_2503_00022_b200 import inputs
+import kvc_testlib as TL
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2503_00022_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+class GpuPass:
+    """Runs the whole pass for a workload on cuda:0, drawing and uploading one layer at a time."""
+
+    def __init__(self, B, w, keep_layers=()):
+        import torch
+        from concurrent.futures import ThreadPoolExecutor
+        self.B, self.w = B, w
+        dev = self.dev = torch.device("cuda:0")
+        tq = {inputs.BF16: torch.bfloat16, inputs.FP32: torch.float32}[w.qk_dtype]
+        tc = {inputs.BF16: torch.bfloat16, inputs.FP16: torch.float16, inputs.FP32: torch.float32}[w.cache_dtype]
+        T = w.total_tokens
+        self.q = torch.empty((w.n_layers, T, w.n_q_heads, w.head_dim), dtype=tq, device=dev)
+        self.k = torch.empty((w.n_layers, T, w.n_kv_heads, w.head_dim), dtype=tq, device=dev)
+        self.kc = torch.empty((w.n_layers, T, w.n_kv_heads, w.head_dim), dtype=tc, device=dev)
+        self.vc = torch.empty((w.n_layers, T, w.n_kv_heads, w.head_dim), dtype=tc, device=dev)
+        self.host = {}
+
+        def one(layer):
+            li = inputs.layer_inputs(w, layer)
+            if layer in keep_layers:
+                self.host[layer] = li
+            return layer, li
+
+        with ThreadPoolExecutor(max_workers=8) as ex:
+            for layer, li in ex.map(one, range(w.n_layers)):
+                self.q[layer].copy_(TL.torch_storage(li.q, w.qk_dtype, dev))
+                self.k[layer].copy_(TL.torch_storage(li.k, w.qk_dtype, dev))
+                self.kc[layer].copy_(TL.torch_storage(li.k_cache, w.cache_dtype, dev))
+                self.vc[layer].copy_(TL.torch_storage(li.v_cache, w.cache_dtype, dev))
+        self.prob = B.Problem(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, causal=w.causal, device=dev)
+        self.b_imp, self.b_rep = w.budgets()
+        self.cp = B.CompressionPass(self.prob, self.b_imp[None, :], self.b_rep[None, :], cache_dtype=tc)
+        self.cp.run(self.q, self.k, self.kc, self.vc)
+        torch.cuda.synchronize()
+        self.cp.check_status()
+        self.scores = self.cp.scores.cpu().numpy()
+        self.lse = self.cp.lse.cpu().numpy()
+
+    # ---- properties that hold at any size -----------------------------------------------------
+    def check_invariants(self):
+        w, cp = self.w, self.cp
+        cu = w.cu_seqlens
+        assert np.isfinite(self.scores).all() and (self.scores >= 0).all()
+        for s, L in enumerate(w.seqlens):
+            tot = self.scores[:, :, cu[s]:cu[s + 1]].astype(np.float64).sum(axis=2)
+            np.testing.assert_allclose(tot, float(L), rtol=2e-4)          # sum_t c_h(t) = number of queries
+        idx = cp.idx.cpu().numpy()
+        kind = cp.kind.cpu().numpy()
+        for l in range(w.n_layers):
+            for s, L in enumerate(w.seqlens):
+                seg = l * w.n_seqs + s
+                lo, hi = int(cp.cu_kept_host[seg]), int(cp.cu_kept_host[seg + 1])
+                B_tot = min(int(self.b_imp[s] + self.b_rep[s]), L)
+                assert hi - lo == B_tot
+                ids = idx[lo:hi]
+                assert ids[0] >= 0 and ids[-1] < L and np.all(np.diff(ids) > 0)
+                if B_tot < L:
+                    assert int(kind[lo:hi].sum()) == int(self.b_rep[s])
+
+    # ---- the oracle's selection on the GPU's scores reproduces the GPU's selection --------------
+    def check_selection_consistency(self, layers):
+        w, cp = self.w, self.cp
+        cu = w.cu_seqlens
+        sigs = cp.sigs.cpu().numpy().view(np.uint32)
+        theta = cp.theta.cpu().numpy()
+        for l in layers:
+            ref = TL.oracle_select_layer(w, self.scores[l], self.b_imp, self.b_rep)
+            for s in range(w.n_seqs):
+                np.testing.assert_array_equal(theta[l, s], ref[s]["theta"])
+                np.testing.assert_array_equal(sigs[l, cu[s]:cu[s + 1]], ref[s]["sig"])
+                np.testing.assert_array_equal(cp.kept(l, s), ref[s]["idx"].astype(np.int32))
+
+    def check_compaction(self, layers):
+        import torch
+        w, cp = self.w, self.cp
+        cu = w.cu_seqlens
+        for l in layers:
+            li = self.host[l]
+            for s in range(w.n_seqs):
+                ids = cp.kept(l, s)
+                seg = l * w.n_seqs + s
+                lo = int(cp.cu_kept_host[seg]) - int(cp.cu_kept_host[l * w.n_seqs])
+                for out, cache in ((cp.k_out, li.k_cache), (cp.v_out, li.v_cache)):
+                    got = out[l, lo:lo + len(ids)].contiguous().view(torch.uint8).cpu().numpy()
+                    assert got.tobytes() == O.compact(cache[cu[s]:cu[s + 1]], ids).tobytes()
+
+    # ---- scores against the oracle -----------------------------------------------------------------
+    def check_scores_heads(self, layer, heads, seqs=None):
+        """Complete column sums and lse of some query heads of one layer."""
+        w = self.w
+        cu = w.cu_seqlens
+        li = self.host[layer]
+        G = w.n_q_heads // w.n_kv_heads
+        for s in (range(w.n_seqs) if seqs is None else seqs):
+            a, b = int(cu[s]), int(cu[s + 1])
+            q = inputs.widen(li.q[a:b][:, heads], w.qk_dtype)
+            k = inputs.widen(li.k[a:b][:, [h // G for h in heads]], w.qk_dtype)
+            c, lse = O.scores(q, k, w.causal)
+            g = self.scores[layer][heads][:, a:b]
+            ok = TL.within_score_tolerance(g, c)
+            assert ok.all(), (w.name, layer, s, np.argwhere(~ok)[:4], g[~ok][:4], c[~ok][:4])
+            np.testing.assert_allclose(self.lse[layer][heads][:, a:b], lse, rtol=0, atol=3e-4)
+        return True
+
+    def check_scores_tail(self, layer, heads, seq, n_rows):
+        """Long sequence: the last n_rows queries give the complete column sums of the last n_rows keys."""
+        w = self.w
+        cu = w.cu_seqlens
+        li = self.host[layer]
+        G = w.n_q_heads // w.n_kv_heads
+        a, b = int(cu[seq]), int(cu[seq + 1])
+        L = b - a
+        q = inputs.widen(li.q[a:b][:, heads], w.qk_dtype)
+        k = inputs.widen(li.k[a:b][:, [h // G for h in heads]], w.qk_dtype)
+        c, lse = O.scores(q, k, True, rows=(L - n_rows, L))
+        g = self.scores[layer][heads][:, b - n_rows:b]
+        ok = TL.within_score_tolerance(g, c[:, L - n_rows:])
+        assert ok.all(), (w.name, layer, np.argwhere(~ok)[:4])
+        np.testing.assert_allclose(self.lse[layer][heads][:, b - n_rows:b], lse[:, L - n_rows:], rtol=0, atol=3e-4)
+
+    def check_lse_rows(self, layer, heads, seq, row_starts, n=16):
+        w = self.w
+        cu = w.cu_seqlens
+        li = self.host[layer]
+        G = w.n_q_heads // w.n_kv_heads
+        a, b = int(cu[seq]), int(cu[seq + 1])
+        q = inputs.widen(li.q[a:b][:, heads], w.qk_dtype)
+        k = inputs.widen(li.k[a:b][:, [h // G for h in heads]], w.qk_dtype)
+        for j0 in row_starts:
+            _, lse = O.scores(q, k, True, rows=(j0, j0 + n))
+            np.testing.assert_allclose(self.lse[layer][heads][:, a + j0:a + j0 + n], lse[:, j0:j0 + n], rtol=0, atol=3e-4)
+
+    # ---- end to end against the oracle's own scores (one layer, all heads) -------------------------
+    def check_end_to_end(self, layer):
+        w, cp = self.w, self.cp
+        cu = w.cu_seqlens
+        li = self.host[layer]
+        c, _ = TL.oracle_scores_layer(w, li)
+        ok = TL.within_score_tolerance(self.scores[layer], c)
+        assert ok.all(), (w.name, layer, np.argwhere(~ok)[:4])
+        o32 = O.to_scores32(c)
+        ref = TL.oracle_select_layer(w, o32, self.b_imp, self.b_rep)
+        sigs = cp.sigs.cpu().numpy().view(np.uint32)
+        exact = 0
+        for s, L in enumerate(w.seqlens):
+            a, b = int(cu[s]), int(cu[s + 1])
+            Hq = w.n_q_heads
+            # (ii) signature bits may differ only where the oracle score is within tolerance of theta_h
+            gb = O.unpack_bits(sigs[layer, a:b], Hq)
+            ob = O.unpack_bits(ref[s]["sig"], Hq)
+            th = ref[s]["theta"].astype(np.float64)
+            for t, h in np.argwhere(gb != ob):
+                # |s_o - theta_o| <= |s_o - s_g| + |theta_g - theta_o|: twice the score tolerance (plus slack)
+                assert abs(float(o32[h, a + t]) - th[h]) <= 2.5 * (TL.SCORE_ATOL + TL.SCORE_RTOL * abs(th[h])), (s, t, h)
+            # (i) important sets may differ only for tokens whose oracle importance is near the cut
+            I_o = O.importance(np.ascontiguousarray(o32[:, a:b]), w.n_kv_heads)
+            bi = int(self.b_imp[s])
+            imp_o = set(O.top_important(I_o, bi).tolist())
+            I_g = O.importance(np.ascontiguousarray(self.scores[layer][:, a:b]), w.n_kv_heads)
+            imp_g = set(O.top_important(I_g, bi).tolist())
+            if bi > 0 and bi < L:
+                cut = np.sort(I_o)[::-1][bi - 1]
+                for t in imp_o ^ imp_g:
+                    assert abs(I_o[t] - cut) <= 2.5 * (Hq * TL.SCORE_ATOL + TL.SCORE_RTOL * cut), (s, t)
+            same_inputs = np.array_equal(gb, ob) and imp_o == imp_g
+            if same_inputs:                      # (iv) then the kept set and the reduced cache match exactly
+                np.testing.assert_array_equal(cp.kept(layer, s), ref[s]["idx"].astype(np.int32))
+                exact += 1
+        return exact
+
+
+def test_cfg1_small_fp32_end_to_end(B):
+    w = inputs.paper_workloads()["cfg1_small_fp32"]
+    gp = GpuPass(B, w, keep_layers=(0,))
+    gp.check_invariants()
+    gp.check_selection_consistency([0])
+    gp.check_compaction([0])
+    gp.check_end_to_end(0)
+
+
+def test_cfg2_llama2_layer_4k_end_to_end(B):
+    w = inputs.paper_workloads()["cfg2_llama2_layer_4k"]
+    gp = GpuPass(B, w, keep_layers=(0,))
+    gp.check_invariants()
+    gp.check_selection_consistency([0])
+    gp.check_compaction([0])
+    gp.check_end_to_end(0)
+
+
+def test_cfg3_llama2_32l_8k_full_size(B):
+    w = inputs.paper_workloads()["cfg3_llama2_32l_8k"]
+    gp = GpuPass(B, w, keep_layers=(0, 15, 31))
+    gp.check_invariants()
+    gp.check_selection_consistency(range(w.n_layers))
+    gp.check_compaction([0, 31])
+    gp.check_end_to_end(0)                                   # all 32 heads of layer 0
+    gp.check_scores_heads(15, [0, 13, 31])
+    gp.check_scores_heads(31, [5, 22])
+
+
+def test_cfg4_llama3_gqa_32k_full_size(B):
+    w = inputs.paper_workloads()["cfg4_llama3_gqa_32k"]
+    gp = GpuPass(B, w, keep_layers=(0, 31))
+    gp.check_invariants()
+    gp.check_selection_consistency([0, 9, 31])
+    gp.check_compaction([31])
+    heads = [0, 3, 4, 31]                                    # two heads of one KV group, two others
+    gp.check_scores_tail(0, heads, 0, 768)
+    gp.check_scores_tail(31, heads, 0, 300)
+    gp.check_lse_rows(0, heads, 0, [0, 127, 128, 5000, 16383, 30000])
+
+
+def test_cfg5_ragged_batch16_full_size(B):
+    w = inputs.paper_workloads()["cfg5_ragged_batch16"]
+    gp = GpuPass(B, w, keep_layers=(0, 31))
+    gp.check_invariants()
+    gp.check_selection_consistency([0, 31])
+    gp.check_compaction([0])
+    gp.check_scores_heads(0, [0, 17, 31])                    # every sequence of the batch
+    gp.check_scores_heads(31, [8], seqs=[0, 7, 15])

@@ -91,6 +91,19 @@ def test_gqa_equals_mha_with_repeated_key_heads():
     np.testing.assert_array_equal(c_gqa, c_mha)
 
 
+def test_row_range_gives_complete_tail_columns():
+    L, Hq, Hkv, D = 90, 4, 2, 16
+    q, k = _rand_qk(L, Hq, Hkv, D, 19)
+    c, lse = O.scores(q, k, True)
+    for j0, j1 in ((60, 90), (0, 90), (33, 34)):
+        cp, lp = O.scores(q, k, True, rows=(j0, j1))
+        A = O.attention_matrix(q, k, True)
+        np.testing.assert_allclose(cp, A[:, j0:j1, :].sum(axis=1), rtol=1e-12, atol=1e-15)
+        np.testing.assert_array_equal(lp[:, j0:j1], lse[:, j0:j1])
+        if j1 == L:
+            np.testing.assert_array_equal(cp[:, j0:], c[:, j0:])       # keys >= j0 are only seen by rows >= j0
+
+
 def test_scale_and_normalize():
     L, H, D = 20, 2, 8
     q, k = _rand_qk(L, H, H, D, 13)
