@@ -31,8 +31,12 @@ namespace {
 
 constexpr int kTile = 128;               // rows of both operands per tile
 constexpr int kStages = 2;               // ring depth of the streamed operand
-constexpr int kThreads = 320;
+#ifndef KVC_EPI_GROUPS
+#define KVC_EPI_GROUPS 2
+#endif
+constexpr int kGroups = KVC_EPI_GROUPS;  // epilogue groups of 128 threads; tile i goes to group i % kGroups
 constexpr int kEpiThreads = 128;         // per epilogue group
+constexpr int kThreads = 64 + kGroups * kEpiThreads;
 constexpr uint32_t kTmemCols = 256;      // two 128-column fp32 accumulators
 constexpr uint32_t kSpinLimit = 1u << 20;
 
@@ -102,21 +106,6 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 32 consecutive fp32 columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
 __device__ __forceinline__ void named_bar_sync(int id, int n) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
 }
@@ -124,6 +113,134 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// 2^x on the FMA pipe for x <= ~0 (any magnitude): round-to-nearest split x = n + f, f in [-0.5, 0.5],
+// cubic minimax polynomial for 2^f (relative error 7.5e-5), exponent bits of n added to the result.
+// The special-function unit delivers 16 ex2 per clock per SM and is the busiest unit of both sweeps;
+// sending a fixed share of the exponentials down this path takes load off it.
+__device__ __forceinline__ float exp2_poly(float x) {
+  x = fmaxf(x, -125.f);                              // keeps the result a normal number (also maps -inf)
+  const float t = x + 12582912.f;                    // 1.5 * 2^23: the integer part lands in the low mantissa bits
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(f, 0.0551716648f, 0.2426111251f);
+  p = fmaf(p, f, 0.6932609677f);
+  p = fmaf(p, f, 0.9999280572f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+#ifndef KVC_POLY_PER8
+#define KVC_POLY_PER8 2                              // of every 8 exponentials, this many use exp2_poly
+#endif
+__host__ __device__ constexpr bool poly_slot(int i) {
+  return ((i % 8 + 1) * KVC_POLY_PER8) / 8 > ((i % 8) * KVC_POLY_PER8) / 8;
+}
+template <int I>
+__device__ __forceinline__ float exp2_mix(float x) {
+  if constexpr (poly_slot(I)) return exp2_poly(x); else return ex2(x);
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// 16 consecutive fp32 columns of this thread's TMEM lane (asynchronous: see tmem_wait16)
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+// Waits for every TMEM load of this thread.  The registers are listed as read-write operands so that
+// no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_wait16(uint32_t (&v)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                 "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+               :: "memory");
+}
+
+// Streams the 128 columns of one accumulator through two 16-column register buffers: the load of the next
+// piece is in flight while the current one is processed.  `release` runs once the last load has landed.
+template <class Piece, class Release>
+__device__ __forceinline__ void sweep_tile(uint32_t taddr, Piece&& piece, Release&& release) {
+  uint32_t va[16], vb[16];
+  tmem_ld16(taddr, va);
+  tmem_wait16(va);
+#pragma unroll
+  for (int p = 0; p < 8; p += 2) {
+    tmem_ld16(taddr + (p + 1) * 16, vb);
+    piece(va, p);
+    tmem_wait16(vb);
+    if (p == 6) release();
+    if (p < 6) tmem_ld16(taddr + (p + 2) * 16, va);
+    piece(vb, p + 1);
+    if (p < 6) tmem_wait16(va);
+  }
+}
+
+// ---- sweep 2: 16 columns (queries) of this thread's key row -------------------------------------
+template <bool kDiag>
+__device__ __forceinline__ void colsum_piece(const uint32_t (&v)[16], const float* lse16, float scale, int r, int c0,
+                                             float (&acc)[4]) {
+  const float4* l4 = reinterpret_cast<const float4*>(lse16);
+#pragma unroll
+  for (int c4 = 0; c4 < 4; ++c4) {
+    const float4 l = l4[c4];
+    float e0, e1, e2, e3;
+    if (c4 == 0) {
+      e0 = exp2_mix<0>(fmaf(__uint_as_float(v[0]), scale, -l.x)); e1 = exp2_mix<1>(fmaf(__uint_as_float(v[1]), scale, -l.y));
+      e2 = exp2_mix<2>(fmaf(__uint_as_float(v[2]), scale, -l.z)); e3 = exp2_mix<3>(fmaf(__uint_as_float(v[3]), scale, -l.w));
+    } else if (c4 == 1) {
+      e0 = exp2_mix<4>(fmaf(__uint_as_float(v[4]), scale, -l.x)); e1 = exp2_mix<5>(fmaf(__uint_as_float(v[5]), scale, -l.y));
+      e2 = exp2_mix<6>(fmaf(__uint_as_float(v[6]), scale, -l.z)); e3 = exp2_mix<7>(fmaf(__uint_as_float(v[7]), scale, -l.w));
+    } else if (c4 == 2) {
+      e0 = exp2_mix<0>(fmaf(__uint_as_float(v[8]), scale, -l.x)); e1 = exp2_mix<1>(fmaf(__uint_as_float(v[9]), scale, -l.y));
+      e2 = exp2_mix<2>(fmaf(__uint_as_float(v[10]), scale, -l.z)); e3 = exp2_mix<3>(fmaf(__uint_as_float(v[11]), scale, -l.w));
+    } else {
+      e0 = exp2_mix<4>(fmaf(__uint_as_float(v[12]), scale, -l.x)); e1 = exp2_mix<5>(fmaf(__uint_as_float(v[13]), scale, -l.y));
+      e2 = exp2_mix<6>(fmaf(__uint_as_float(v[14]), scale, -l.z)); e3 = exp2_mix<7>(fmaf(__uint_as_float(v[15]), scale, -l.w));
+    }
+    if constexpr (kDiag) {                          // causal: the query (column) must not precede the key (row)
+      const int c = c0 + 4 * c4;
+      e0 = c + 0 >= r ? e0 : 0.f; e1 = c + 1 >= r ? e1 : 0.f;
+      e2 = c + 2 >= r ? e2 : 0.f; e3 = c + 3 >= r ? e3 : 0.f;
+    }
+    acc[0] += e0; acc[1] += e1; acc[2] += e2; acc[3] += e3;
+  }
+}
+
+// ---- sweep 1: 16 columns (keys) of this thread's query row; online max / sum in the log2 domain ----
+template <bool kMasked>
+__device__ __forceinline__ void lse_piece(const uint32_t (&v)[16], float scale, int c_lim, float& m, float& sum) {
+  float x[16];
+#pragma unroll
+  for (int c = 0; c < 16; ++c) x[c] = __uint_as_float(v[c]);
+  if constexpr (kMasked) {
+    if (c_lim <= 0) return;                         // nothing of this piece belongs to the row
+#pragma unroll
+    for (int c = 0; c < 16; ++c) x[c] = c < c_lim ? x[c] : __int_as_float(0xFF800000);
+  }
+  const float m0 = max3(x[0], x[1], x[2]), m1 = max3(x[3], x[4], x[5]), m2 = max3(x[6], x[7], x[8]);
+  const float m3 = max3(x[9], x[10], x[11]), m4 = max3(x[12], x[13], x[14]);
+  const float cmax = fmaxf(max3(m0, m1, m2), max3(m3, m4, x[15]));
+  const float m_new = fmaxf(m, cmax * scale);
+  if (m_new > m) { sum *= ex2(m - m_new); m = m_new; }
+  float s0, s1, s2, s3;
+  s0 = exp2_mix<0>(fmaf(x[0], scale, -m)); s1 = exp2_mix<1>(fmaf(x[1], scale, -m));
+  s2 = exp2_mix<2>(fmaf(x[2], scale, -m)); s3 = exp2_mix<3>(fmaf(x[3], scale, -m));
+  s0 += exp2_mix<4>(fmaf(x[4], scale, -m)); s1 += exp2_mix<5>(fmaf(x[5], scale, -m));
+  s2 += exp2_mix<6>(fmaf(x[6], scale, -m)); s3 += exp2_mix<7>(fmaf(x[7], scale, -m));
+  s0 += exp2_mix<0>(fmaf(x[8], scale, -m)); s1 += exp2_mix<1>(fmaf(x[9], scale, -m));
+  s2 += exp2_mix<2>(fmaf(x[10], scale, -m)); s3 += exp2_mix<3>(fmaf(x[11], scale, -m));
+  s0 += exp2_mix<4>(fmaf(x[12], scale, -m)); s1 += exp2_mix<5>(fmaf(x[13], scale, -m));
+  s2 += exp2_mix<6>(fmaf(x[14], scale, -m)); s3 += exp2_mix<7>(fmaf(x[15], scale, -m));
+  sum += (s0 + s1) + (s2 + s3);
 }
 
 // Shared-memory matrix descriptor of a K-major tile stored as 128-byte rows with the 128B swizzle
@@ -225,8 +342,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Shape& s = a.s;
   const int n_lh = s.n_layers * s.Hq;
+  // Block order: all tile-rows of one (layer, head) are adjacent, heaviest first, so the CTAs that run
+  // at the same time stream the same few heads' Q/K and those stay in L2.
+#ifdef KVC_RANK_MAJOR
   const int lh = blockIdx.x % n_lh;
   const int rank = blockIdx.x / n_lh;
+#else
+  const int lh = blockIdx.x / a.n_items;
+  const int rank = blockIdx.x - lh * a.n_items;
+#endif
   const int layer = lh / s.Hq, h = lh - layer * s.Hq;
   const int hk = h / s.G;
 
@@ -322,7 +446,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
   } else {
     // ------------------------------ epilogue groups ------------------------------
-    const int g = (warp - 2) >> 2;                 // group 0 takes even tiles, group 1 odd tiles
+    const int g = (warp - 2) >> 2;                 // epilogue group of this warp
     const int quarter = warp & 3;                  // TMEM lanes this warp may read
     const int r = quarter * 32 + lane;             // row of the accumulator tile = TMEM lane
     const int gtid = r;                            // index inside the group (0..127)
@@ -332,111 +456,85 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     if constexpr (kColsum) {
       const float* lse_row = a.lse + ((size_t)layer * s.Hq + h) * s.T + t0;
-      float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+      const float inf = __int_as_float(0x7F800000);
+      auto load_lse = [&](int it) {                 // lse2 of this thread's query of streamed tile `it` (+inf past the end)
+        const int j = (first_stream + it) * kTile + gtid;
+        return (it < n_iter && j < L) ? __ldg(lse_row + j) * a.lse_mul : inf;
+      };
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      float lse_next = load_lse(g);
       int n_mine = 0;
-      for (int it = g; it < n_iter; it += 2, ++n_mine) {
-        const int q0 = (first_stream + it) * kTile;
+      for (int it = g; it < n_iter; it += kGroups, ++n_mine) {
+        const int b = it & 1;                       // TMEM accumulator of this tile
         float* lse_buf = aux->lse_sh[g][n_mine & 1];
-        {
-          const int j = q0 + gtid;
-          lse_buf[gtid] = j < L ? __ldg(lse_row + j) * a.lse_mul : __int_as_float(0x7F800000);
-        }
+        lse_buf[gtid] = lse_next;
+        lse_next = load_lse(it + kGroups);          // in flight while this tile is processed
         named_bar_sync(1 + g, kEpiThreads);
         // after a failed wait the loop keeps running (every thread must reach every named barrier) but
         // touches neither barriers nor TMEM; `ok` is made warp-uniform because tcgen05.ld is warp-wide
-        if (ok) ok = mbar_wait(smem_u32(&aux->acc_full[g]), n_mine & 1, abort_flag);
+        if (ok) ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it >> 1) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) continue;
         tc_fence_after();
-        const bool diag = s.causal && it == 0;
-#pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(t_lane + g * kTile + ch * 32, v);
-          tmem_ld_wait();
-          if (ch == 3) {                          // accumulator drained: hand the buffer back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&aux->acc_empty[g]));
-          }
-          const float4* l4 = reinterpret_cast<const float4*>(lse_buf + ch * 32);
-#pragma unroll
-          for (int c4 = 0; c4 < 8; ++c4) {
-            const float4 l = l4[c4];
-            float e0 = ex2(fmaf(__uint_as_float(v[4 * c4 + 0]), scale, -l.x));
-            float e1 = ex2(fmaf(__uint_as_float(v[4 * c4 + 1]), scale, -l.y));
-            float e2 = ex2(fmaf(__uint_as_float(v[4 * c4 + 2]), scale, -l.z));
-            float e3 = ex2(fmaf(__uint_as_float(v[4 * c4 + 3]), scale, -l.w));
-            if (diag) {                           // causal: query (column) must not precede key (row)
-              const int c = ch * 32 + 4 * c4;
-              e0 = c + 0 >= r ? e0 : 0.f; e1 = c + 1 >= r ? e1 : 0.f;
-              e2 = c + 2 >= r ? e2 : 0.f; e3 = c + 3 >= r ? e3 : 0.f;
-            }
-            acc0 += e0; acc1 += e1; acc2 += e2; acc3 += e3;
-          }
-        }
+        auto release = [&]() {                      // accumulator drained: hand it back to the MMA warp
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&aux->acc_empty[b]));
+        };
+        const uint32_t t_acc = t_lane + b * kTile;
+        if (s.causal && it == 0)
+          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
+        else
+          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
       }
-      const float acc = (acc0 + acc1) + (acc2 + acc3);
-      if (g == 1) aux->part[0][r] = acc;
-      named_bar_sync(3, 2 * kEpiThreads);
+      float total = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+      if constexpr (kGroups == 2) {
+        if (g == 1) aux->part[0][r] = total;
+        named_bar_sync(3, 2 * kEpiThreads);
+        if (g == 0) total += aux->part[0][r];
+      }
       if (g == 0 && ok && !*abort_flag) {
         const int t = my_tile * kTile + r;
         if (t < L) {
-          float total = acc + aux->part[0][r];
           if (a.normalize) total = total / (float)L;
           a.scores[((size_t)layer * s.Hq + h) * s.T + t0 + t] = total;
         }
       }
     } else {
       float m = __int_as_float(0xFF800000), sum = 0.f;        // running max (log2 domain) and sum of this row
-      int n_mine = 0;
-      for (int it = g; it < n_iter; it += 2, ++n_mine) {
-        ok = mbar_wait(smem_u32(&aux->acc_full[g]), n_mine & 1, abort_flag);
+      for (int it = g; it < n_iter; it += kGroups) {
+        const int b = it & 1;
+        ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it >> 1) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         tc_fence_after();
-        const bool diag = s.causal && it == my_tile;
-        const int n_valid = s.causal ? kTile : min(kTile, L - it * kTile);    // keys of this tile inside the sequence
-#pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(t_lane + g * kTile + ch * 32, v);
-          tmem_ld_wait();
-          if (ch == 3) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&aux->acc_empty[g]));
-          }
-          const int c_lim = min(diag ? r + 1 : kTile, n_valid) - ch * 32;       // columns [0, c_lim) of the chunk count
-          if (c_lim < 32) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) v[c] = c < c_lim ? v[c] : 0xFF800000u;
-          }
-          float cmax = __uint_as_float(v[0]);
-#pragma unroll
-          for (int c = 1; c < 32; ++c) cmax = fmaxf(cmax, __uint_as_float(v[c]));
-          const float m_new = fmaxf(m, cmax * scale);
-          if (m_new > m) { sum *= ex2(m - m_new); m = m_new; }
-          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-          for (int c = 0; c < 32; c += 4) {
-            s0 += ex2(fmaf(__uint_as_float(v[c + 0]), scale, -m));
-            s1 += ex2(fmaf(__uint_as_float(v[c + 1]), scale, -m));
-            s2 += ex2(fmaf(__uint_as_float(v[c + 2]), scale, -m));
-            s3 += ex2(fmaf(__uint_as_float(v[c + 3]), scale, -m));
-          }
-          if (c_lim > 0) sum += (s0 + s1) + (s2 + s3);
+        auto release = [&]() {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&aux->acc_empty[b]));
+        };
+        const uint32_t t_acc = t_lane + b * kTile;
+        // keys of this tile that count for this row: up to the diagonal (causal) and inside the sequence
+        const int n_valid = s.causal ? (it == my_tile ? r + 1 : kTile) : min(kTile, L - it * kTile);
+        if (__any_sync(0xFFFFFFFFu, n_valid < kTile))
+          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, n_valid - p * 16, m, sum); }, release);
+        else
+          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, 16, m, sum); }, release);
+      }
+      if constexpr (kGroups == 2) {
+        if (g == 1) { aux->part[0][r] = m; aux->part[1][r] = sum; }
+        named_bar_sync(3, 2 * kEpiThreads);
+        if (g == 0) {                               // merge the other group's (max, sum)
+          const float m1 = aux->part[0][r], sum1 = aux->part[1][r];
+          const float big = fmaxf(m, m1);
+          sum = sum * ex2(m - big) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
+          m = big;
         }
       }
-      if (g == 1) { aux->part[0][r] = m; aux->part[1][r] = sum; }
-      named_bar_sync(3, 2 * kEpiThreads);
       if (g == 0 && ok && !*abort_flag) {
         const int j = my_tile * kTile + r;
         if (j < L) {
-          const float m1 = aux->part[0][r], sum1 = aux->part[1][r];
-          const float big = fmaxf(m, m1);
-          const float tot = sum * ex2(m - big) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
-          const float lse2 = big + log2f(tot);
+          const float lse2 = m + log2f(sum);
           const size_t o = ((size_t)layer * s.Hq + h) * s.T + t0 + j;
           a.lse2_out[o] = lse2;
           if (a.lse_nat_out) a.lse_nat_out[o] = lse2 * 0.69314718055994530942f;
