@@ -30,14 +30,19 @@ namespace kvc {
 namespace {
 
 constexpr int kTile = 128;               // rows of both operands per tile
-constexpr int kStages = 2;               // ring depth of the streamed operand
 #ifndef KVC_EPI_GROUPS
 #define KVC_EPI_GROUPS 2
 #endif
 constexpr int kGroups = KVC_EPI_GROUPS;  // epilogue groups of 128 threads; tile i goes to group i % kGroups
 constexpr int kEpiThreads = 128;         // per epilogue group
 constexpr int kThreads = 64 + kGroups * kEpiThreads;
-constexpr uint32_t kTmemCols = 256;      // two 128-column fp32 accumulators
+constexpr int kBufs = kGroups < 2 ? 2 : kGroups;         // 128-column fp32 accumulators in TMEM; tile i uses buffer i % kBufs
+constexpr uint32_t kTmemCols = kBufs * 128;
+constexpr int kCtasPerSm = kGroups > 2 ? 1 : 2;
+#ifndef KVC_STAGES
+#define KVC_STAGES (kGroups > 2 ? 5 : 2)
+#endif
+constexpr int kStages = KVC_STAGES;      // ring depth of the streamed operand
 constexpr uint32_t kSpinLimit = 1u << 20;
 
 // ------------------------------------------------------------------------------------------------
@@ -309,7 +314,7 @@ struct SmemLayout {
   static constexpr int kFixedOff = 0;
   static constexpr int kRingOff = kTileBytes;
   static constexpr int kAuxOff = kRingOff + kStages * kTileBytes;
-  static constexpr int kAuxBytes = 4096;
+  static constexpr int kAuxBytes = 12288;
   static constexpr int kTotal = kAuxOff + kAuxBytes + 1024;  // + slack to align the base to 1024
 };
 
@@ -317,18 +322,18 @@ struct Aux {                         // lives at kAuxOff
   unsigned long long full[kStages];
   unsigned long long empty[kStages];
   unsigned long long fixed_full;
-  unsigned long long acc_full[2];
-  unsigned long long acc_empty[2];
+  unsigned long long acc_full[kBufs];
+  unsigned long long acc_empty[kBufs];
   unsigned long long drain;
   uint32_t tmem_base;
   int abort_flag;
   int item[4];                       // seq, tile, n_tiles
-  alignas(16) float lse_sh[2][2][kTile];         // [group][buffer][query in tile]   (sweep 2)
-  alignas(16) float part[2][kTile];              // group 1 partials handed to group 0
+  alignas(16) float lse_sh[kGroups][2][kTile];   // [group][buffer][query in tile]   (sweep 2)
+  alignas(16) float part[kGroups][2][kTile];     // partials of groups 1.. handed to group 0
 };
 
 template <int D, bool kColsum>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const ScoreArgs a) {
   using SL = SmemLayout<D>;
@@ -341,7 +346,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Shape& s = a.s;
+#ifdef KVC_RANK_MAJOR
   const int n_lh = s.n_layers * s.Hq;
+#endif
   // Block order: all tile-rows of one (layer, head) are adjacent, heaviest first, so the CTAs that run
   // at the same time stream the same few heads' Q/K and those stay in L2.
 #ifdef KVC_RANK_MAJOR
@@ -364,7 +371,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&aux->full[i]), 1); mbar_init(smem_u32(&aux->empty[i]), 1); }
       mbar_init(smem_u32(&aux->fixed_full), 1);
       mbar_init(smem_u32(&aux->drain), 1);
-      for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&aux->acc_full[i]), 1); mbar_init(smem_u32(&aux->acc_empty[i]), 4); }
+      for (int i = 0; i < kBufs; ++i) { mbar_init(smem_u32(&aux->acc_full[i]), 1); mbar_init(smem_u32(&aux->acc_empty[i]), 4); }
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -423,9 +430,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       constexpr uint32_t idesc = make_idesc(kTile, kTile);
       bool ok = mbar_wait(smem_u32(&aux->fixed_full), 0, abort_flag);
       for (int it = 0; ok && it < n_iter; ++it) {
-        const int st = it % kStages, b = it & 1;
+        const int st = it % kStages, b = it % kBufs;
         ok = mbar_wait(smem_u32(&aux->full[st]), (it / kStages) & 1, abort_flag) &&
-             mbar_wait(smem_u32(&aux->acc_empty[b]), ((it >> 1) & 1) ^ 1, abort_flag);
+             mbar_wait(smem_u32(&aux->acc_empty[b]), ((it / kBufs) & 1) ^ 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + b * kTile;
@@ -465,14 +472,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       float lse_next = load_lse(g);
       int n_mine = 0;
       for (int it = g; it < n_iter; it += kGroups, ++n_mine) {
-        const int b = it & 1;                       // TMEM accumulator of this tile
+        const int b = it % kBufs;                   // TMEM accumulator of this tile
         float* lse_buf = aux->lse_sh[g][n_mine & 1];
         lse_buf[gtid] = lse_next;
         lse_next = load_lse(it + kGroups);          // in flight while this tile is processed
         named_bar_sync(1 + g, kEpiThreads);
         // after a failed wait the loop keeps running (every thread must reach every named barrier) but
         // touches neither barriers nor TMEM; `ok` is made warp-uniform because tcgen05.ld is warp-wide
-        if (ok) ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it >> 1) & 1, abort_flag);
+        if (ok) ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it / kBufs) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) continue;
         tc_fence_after();
@@ -488,10 +495,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
       }
       float total = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-      if constexpr (kGroups == 2) {
-        if (g == 1) aux->part[0][r] = total;
-        named_bar_sync(3, 2 * kEpiThreads);
-        if (g == 0) total += aux->part[0][r];
+      if constexpr (kGroups > 1) {
+        if (g > 0) aux->part[g][0][r] = total;
+        named_bar_sync(1 + kGroups, kGroups * kEpiThreads);
+        if (g == 0)
+          for (int o = 1; o < kGroups; ++o) total += aux->part[o][0][r];
       }
       if (g == 0 && ok && !*abort_flag) {
         const int t = my_tile * kTile + r;
@@ -503,8 +511,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     } else {
       float m = __int_as_float(0xFF800000), sum = 0.f;        // running max (log2 domain) and sum of this row
       for (int it = g; it < n_iter; it += kGroups) {
-        const int b = it & 1;
-        ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it >> 1) & 1, abort_flag);
+        const int b = it % kBufs;
+        ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it / kBufs) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -521,14 +529,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         else
           sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, 16, m, sum); }, release);
       }
-      if constexpr (kGroups == 2) {
-        if (g == 1) { aux->part[0][r] = m; aux->part[1][r] = sum; }
-        named_bar_sync(3, 2 * kEpiThreads);
-        if (g == 0) {                               // merge the other group's (max, sum)
-          const float m1 = aux->part[0][r], sum1 = aux->part[1][r];
-          const float big = fmaxf(m, m1);
-          sum = sum * ex2(m - big) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
-          m = big;
+      if constexpr (kGroups > 1) {
+        if (g > 0) { aux->part[g][0][r] = m; aux->part[g][1][r] = sum; }
+        named_bar_sync(1 + kGroups, kGroups * kEpiThreads);
+        if (g == 0) {                               // merge the other groups' (max, sum)
+          for (int o = 1; o < kGroups; ++o) {
+            const float m1 = aux->part[o][0][r], sum1 = aux->part[o][1][r];
+            const float big = fmaxf(m, m1);
+            sum = sum * ex2(m - big) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
+            m = big;
+          }
         }
       }
       if (g == 0 && ok && !*abort_flag) {
@@ -612,7 +622,7 @@ bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorVie
 int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView& Q, const TensorView& K,
                         float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores,
                         float* lse_out, int normalize, int32_t* status, cudaStream_t stream) {
-  static_assert(sizeof(Aux) <= 4096, "aux block too large");
+  static_assert(sizeof(Aux) <= 12288, "aux block too large");
   if (!(scale_log2 > 0.f)) return KVCRUSH_ERR_UNSUPPORTED;
   CUtensorMap mq, mk;
   if (!make_map(&mq, Q, s.D, s.T, s.Hq, s.n_layers) || !make_map(&mk, K, s.D, s.T, s.Hkv, s.n_layers))
