@@ -66,6 +66,30 @@ def algorithmic_work(w: inputs.Workload):
 
 
 # ---------------------------------------------------------------------------------------------
+# multi-process plumbing (one process per GPU; the data path itself has no collective)
+# ---------------------------------------------------------------------------------------------
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("LOCAL_RANK", "0"))
+
+
+def max_over_ranks(value: float, device, world: int) -> float:
+    """Slowest rank's time: what the whole job waits for."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_replica: int, world: int, ms_per_step: float) -> float:
+    """Every rank compresses its own replica of the workload: aggregate prompt tokens per second."""
+    return tokens_per_replica * world / (ms_per_step * 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------
 # clocks
 # ---------------------------------------------------------------------------------------------
 
@@ -192,8 +216,8 @@ def oracle_sample(w: inputs.Workload, max_heads=None):
 
 
 def run_reference(args, w):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    rank, _, _ = dist_env()
+    if rank != 0:                      # under torchrun only rank 0 runs the CPU oracle; the others leave
         return
     from oracle import kvcrush_oracle as O
     O.build_c()
@@ -225,9 +249,7 @@ def run_ours(args, w):
     from paper_2503_00022_b200 import binding as B
     from paper_2503_00022_b200 import build as kbuild
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = dist_env()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
@@ -284,10 +306,7 @@ def run_ours(args, w):
     cp.check_status()
     total_ms = e0.elapsed_time(e1)
     stage_ms = np.asarray([[ev[i][j].elapsed_time(ev[i][j + 1]) for j in range(4)] for i in range(args.steps)]).mean(axis=0)
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev, world)
     ms_per_step = total_ms / args.steps
 
     # ---- end to end through host buffers: H2D of the step's inputs, D2H of the kept set and reduced cache ----
@@ -315,11 +334,7 @@ def run_ours(args, w):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_ms /= e2e_steps
+    e2e_ms = max_over_ranks(e2e_ms, dev, world) / e2e_steps
     nbytes = lambda t: t.numel() * t.element_size()  # noqa: E731
     h2d = nbytes(hq) + nbytes(hk) + (nbytes(hkc) if hkc is not hk else 0) + nbytes(hvc)
     d2h = nbytes(h_idx) + nbytes(h_ko) + nbytes(h_vo)
@@ -360,7 +375,7 @@ def run_ours(args, w):
 
     tokens = w.total_tokens * world
     line = {
-        "metric": METRIC, "value": tokens / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job_value(w.total_tokens, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if w.qk_dtype == inputs.BF16 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
