@@ -125,7 +125,8 @@ int kvcrush_workspace_size(const kvcrush_problem_t* problem, int stage, size_t* 
  *   lse_out_dev optional out, same shape: the row log-sum-exp (natural log);
  *               not written when lse_in_dev is given
  *   impl        KVCRUSH_SCORE_*
- *   workspace   kvcrush_workspace_size(.., KVCRUSH_STAGE_SCORE, ..) bytes
+ *   workspace   kvcrush_workspace_size(.., KVCRUSH_STAGE_SCORE, ..) bytes (always required: it also
+ *               holds the kernels' work counters)
  */
 int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, const kvcrush_tensor_t* K,
                   const float* lse_in_dev, float* scores_dev, float* lse_out_dev, int normalize, int impl,

@@ -46,7 +46,9 @@ int make_view(const kvcrush_tensor_t* t, int head_dim, TensorView* v) {
   return KVCRUSH_OK;
 }
 
-size_t score_ws(const Shape& s) { return round_up((size_t)s.n_layers * s.Hq * s.T * sizeof(float)); }
+size_t score_lse_bytes(const Shape& s) { return round_up((size_t)s.n_layers * s.Hq * s.T * sizeof(float)); }
+// row log-sum-exp of every query + the work counters of the persistent tensor-core kernels
+size_t score_ws(const Shape& s) { return score_lse_bytes(s) + round_up(score_persist_counter_bytes()); }
 size_t signature_ws(const Shape& s) { return round_up((size_t)s.n_layers * s.n_seqs * s.Hq * sizeof(float)); }
 
 }  // namespace
@@ -85,12 +87,10 @@ int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, c
   if (q.dtype != KVCRUSH_BF16 && q.dtype != KVCRUSH_FP32) return KVCRUSH_ERR_UNSUPPORTED;
   if (impl != KVCRUSH_SCORE_AUTO && impl != KVCRUSH_SCORE_SIMT && impl != KVCRUSH_SCORE_TENSOR)
     return KVCRUSH_ERR_INVALID_ARG;
-  float* lse2_ws = nullptr;
-  if (!lse_in_dev) {
-    if (!workspace || workspace_bytes < score_ws(s)) return KVCRUSH_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
-    lse2_ws = static_cast<float*>(workspace);
-  }
+  if (!workspace || workspace_bytes < score_ws(s)) return KVCRUSH_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
+  float* lse2_ws = static_cast<float*>(workspace);
+  int* counters = reinterpret_cast<int*>(static_cast<unsigned char*>(workspace) + score_lse_bytes(s));
   const float scale = problem->softmax_scale != 0.f ? problem->softmax_scale : 1.f / sqrtf((float)s.D);
   const float log2e = 1.4426950408889634f;
   const float scale_log2 = scale * log2e;
@@ -100,8 +100,14 @@ int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, c
   if (impl == KVCRUSH_SCORE_SIMT || !tensor_ok)
     return launch_score_simt(s, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, scores_dev, lse_out_dev, normalize,
                              status_dev, st);
+#ifndef KVC_TENSOR_PERSISTENT
+  (void)counters;
   return launch_score_tensor(s, problem->cu_seqlens_host, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, scores_dev,
                              lse_out_dev, normalize, status_dev, st);
+#else
+  return launch_score_tensor_persistent(s, problem->cu_seqlens_host, q, k, scale_log2, lse_in_dev, log2e, lse2_ws,
+                                        counters, scores_dev, lse_out_dev, normalize, status_dev, st);
+#endif
 }
 
 int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev, const int32_t* sig_keep_dev,

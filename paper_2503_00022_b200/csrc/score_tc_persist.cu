@@ -1,0 +1,459 @@
+// Stage 1, persistent tensor-core kernels: the same two sweeps as score_tc.cu (Algorithm 1 of the paper:
+// row log-sum-exp, then attention column sums) with a work decomposition built to spend less energy per
+// logit tile, because on this part the sweeps run against the board's power limit:
+//
+//   * one CTA per SM lives for the whole launch and pulls work items from an atomic counter, so TMEM
+//     allocation, barrier set-up and pipeline fill are paid once per SM instead of once per item;
+//   * an item is a 256-row block of the stationary operand (two 128-row halves).  Every streamed
+//     128-row tile is multiplied with both halves, which halves the L2 -> shared-memory traffic per logit;
+//   * TMEM holds four 128-column accumulators, two per half, so the tensor core fills one buffer of a half
+//     while an epilogue group drains the other.
+//
+// Roles: warp 0 fetches + decodes items and issues TMA loads; warp 1 (one lane) issues tcgen05.mma;
+// warps 2..17 are four epilogue groups (half x buffer parity) of 128 threads, thread = TMEM lane = one
+// query row (sweep 1) or one key column (sweep 2).  All synchronisation is by mbarriers with bounded
+// waits: a role that gives up sets the CTA's abort flag, every other wait then ends, the CTA reports
+// through the status word, drains its copies, frees TMEM and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace kvc {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kTile = 128;
+constexpr int kBlockRows = 2 * kTile;        // stationary rows per work item
+constexpr int kEpiWarps = 16;
+constexpr int kThreads = 64 + kEpiWarps * 32;
+constexpr int kRing = 4;                     // streamed tiles in flight
+constexpr uint32_t kTmemCols = 512;          // 4 accumulators x 128 fp32 columns
+
+struct PersistArgs {
+  Shape s;
+  float scale_log2;
+  const float* lse;        // sweep 2: row log-sum-exp; value * lse_mul is in the log2 domain
+  float lse_mul;
+  float* lse2_out;         // sweep 1 output (log2 domain), [n_layers][Hq][T]
+  float* lse_nat_out;      // sweep 1: optional natural-log copy
+  float* scores;           // sweep 2 output
+  int normalize;
+  int max_blocks;          // ceil(max_seqlen / 256)
+  int n_items;             // (sequence, 256-row block) pairs of one (layer, head)
+  int total_items;         // n_items * n_layers * Hq
+  int* counter;            // work counter, zero at launch
+  int32_t* status;
+};
+
+template <int D>
+struct PSmem {
+  static constexpr int kTileBytes = kTile * D * 2;
+  static constexpr int kBlockBytes = kTile * 128;
+  static constexpr int kFixedOff = 0;                            // two stationary halves
+  static constexpr int kRingOff = 2 * kTileBytes;
+  static constexpr int kAuxOff = kRingOff + kRing * kTileBytes;
+  static constexpr int kAuxBytes = 10240;
+  static constexpr int kTotal = kAuxOff + kAuxBytes + 1024;
+};
+
+struct PAux {
+  unsigned long long full[kRing], empty[kRing];
+  unsigned long long fixed_full, fixed_empty;
+  unsigned long long acc_full[4], acc_empty[4];       // [half * 2 + parity]
+  unsigned long long item_full[2], item_empty[2];
+  unsigned long long pair_bar[2];                     // both groups of one half (8 warps)
+  unsigned long long group_bar[4];                    // one group (4 warps)
+  unsigned long long drain;
+  uint32_t tmem_base;
+  int abort_flag;
+  int item[2][8];                                     // layer, head, seq, block, n_tiles (layer < 0: no more work)
+  alignas(16) float lse_sh[4][2][kTile];              // [group][buffer][query of the streamed tile]
+  alignas(16) float part[2][2][2][kTile];             // [half][item parity][value][row]
+};
+
+// Geometry of one work item, derived identically by every role.
+template <bool kColsum>
+struct Geo {
+  int layer, h, hk, t0, L, blk, first_stream, n_iter;
+  bool causal, half1;
+  __device__ __forceinline__ Geo(const Shape& s, const int* it) {
+    layer = it[0]; h = it[1]; hk = h / s.G; blk = it[3];
+    const int seq = it[2], n_tiles = it[4];
+    t0 = __ldg(s.cu_seqlens + seq);
+    L = __ldg(s.cu_seqlens + seq + 1) - t0;
+    causal = s.causal != 0;
+    half1 = blk * kBlockRows + kTile < L;                               // does the second half hold any row
+    if (kColsum) {                                                      // stationary keys, streamed query tiles
+      first_stream = causal ? 2 * blk : 0;
+      n_iter = n_tiles - first_stream;
+    } else {                                                            // stationary queries, streamed key tiles
+      first_stream = 0;
+      n_iter = causal ? min(2 * blk + 2, n_tiles) : n_tiles;
+    }
+  }
+  // does streamed tile `it` contribute to half `hf` (causal: the half's own tile index is 2*blk + hf)
+  __device__ __forceinline__ bool active(int hf, int it) const {
+    if (hf == 1 && !half1) return false;
+    if (!causal) return true;
+    return kColsum ? it >= hf : it <= 2 * blk + hf;
+  }
+  __device__ __forceinline__ bool diag(int hf, int it) const {
+    return causal && (kColsum ? it == hf : it == 2 * blk + hf);
+  }
+};
+
+template <int D, bool kColsum>
+__global__ void __launch_bounds__(kThreads, 1)
+score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                     const PersistArgs a) {
+  using SL = PSmem<D>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  PAux* aux = reinterpret_cast<PAux*>(smem + SL::kAuxOff);
+  volatile int* abort_flag = &aux->abort_flag;
+  const uint32_t fixed_addr = smem_u32(smem + SL::kFixedOff);
+  const uint32_t ring_addr = smem_u32(smem + SL::kRingOff);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const Shape& s = a.s;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // a launch that already failed somewhere is not worth finishing
+      aux->abort_flag = *reinterpret_cast<volatile int32_t*>(a.status) != 0;
+      for (int i = 0; i < kRing; ++i) { mbar_init(smem_u32(&aux->full[i]), 1); mbar_init(smem_u32(&aux->empty[i]), 1); }
+      mbar_init(smem_u32(&aux->fixed_full), 1);
+      mbar_init(smem_u32(&aux->fixed_empty), 1);
+      mbar_init(smem_u32(&aux->drain), 1);
+      for (int i = 0; i < 4; ++i) {
+        mbar_init(smem_u32(&aux->acc_full[i]), 1);
+        mbar_init(smem_u32(&aux->acc_empty[i]), 4);
+        mbar_init(smem_u32(&aux->group_bar[i]), 4);
+      }
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(smem_u32(&aux->item_full[i]), 1);
+        mbar_init(smem_u32(&aux->item_empty[i]), 1 + kEpiWarps);
+        mbar_init(smem_u32(&aux->pair_bar[i]), 8);
+      }
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+  } else if (warp == 1) {
+    tmem_alloc(smem_u32(&aux->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = aux->tmem_base;
+  const bool dead = aux->abort_flag != 0;
+
+  const CUtensorMap* map_fixed = kColsum ? &map_k : &map_q;
+  const CUtensorMap* map_stream = kColsum ? &map_q : &map_k;
+
+  if (dead) {
+    // nothing to do
+  } else if (warp == 0) {
+    // ------------------------------ work fetch + TMA producer ------------------------------
+    int n_item = 0, n_stream = 0;
+    int issued_item = 0;              // lane 0: items whose stationary load was issued
+    bool alive = true;
+    while (alive) {
+      const int slot = n_item & 1;
+      int idx = 0;
+      bool ok = true;
+      if (lane == 0) {
+        ok = mbar_wait(smem_u32(&aux->item_empty[slot]), ((n_item >> 1) & 1) ^ 1, abort_flag);
+        if (ok) idx = atomicAdd(a.counter, 1);
+      }
+      ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+      idx = __shfl_sync(0xFFFFFFFFu, idx, 0);
+      if (!ok) break;
+      if (idx >= a.total_items) {
+        if (lane == 0) { aux->item[slot][0] = -1; mbar_arrive(smem_u32(&aux->item_full[slot])); }
+        break;
+      }
+      const int lh = idx / a.n_items, rank = idx - lh * a.n_items;
+      int seq, blk, nblk;
+      decode_item(s.cu_seqlens, s.n_seqs, a.max_blocks, rank, !kColsum, lane, seq, blk, nblk, kBlockRows);
+      if (lane == 0) {
+        int* it = aux->item[slot];
+        it[0] = lh / s.Hq; it[1] = lh - it[0] * s.Hq; it[2] = seq; it[3] = blk;
+        it[4] = (__ldg(s.cu_seqlens + seq + 1) - __ldg(s.cu_seqlens + seq) + kTile - 1) / kTile;
+        mbar_arrive(smem_u32(&aux->item_full[slot]));
+        const Geo<kColsum> g(s, it);
+        const int head_fixed = kColsum ? g.hk : g.h, head_stream = kColsum ? g.h : g.hk;
+        // the stationary buffer is free once every MMA of the previous item has retired
+        ok = mbar_wait(smem_u32(&aux->fixed_empty), (n_item & 1) ^ 1, abort_flag);
+        if (ok) {
+          const int n_half = g.half1 ? 2 : 1;
+          mbar_expect_tx(smem_u32(&aux->fixed_full), n_half * SL::kTileBytes);
+          for (int hf = 0; hf < n_half; ++hf)
+#pragma unroll
+            for (int kb = 0; kb < D / 64; ++kb)
+              tma_load_4d(fixed_addr + hf * SL::kTileBytes + kb * SL::kBlockBytes, map_fixed, smem_u32(&aux->fixed_full),
+                          kb * 64, g.t0 + g.blk * kBlockRows + hf * kTile, head_fixed, g.layer);
+          issued_item = n_item + 1;
+          for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
+            const int rs = n_stream % kRing;
+            ok = mbar_wait(smem_u32(&aux->empty[rs]), ((n_stream / kRing) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(smem_u32(&aux->full[rs]), SL::kTileBytes);
+#pragma unroll
+            for (int kb = 0; kb < D / 64; ++kb)
+              tma_load_4d(ring_addr + rs * SL::kTileBytes + kb * SL::kBlockBytes, map_stream, smem_u32(&aux->full[rs]),
+                          kb * 64, g.t0 + (g.first_stream + i) * kTile, head_stream, g.layer);
+          }
+        }
+      }
+      alive = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+      n_stream = __shfl_sync(0xFFFFFFFFu, n_stream, 0);
+      ++n_item;
+    }
+    if (lane == 0 && *abort_flag) {
+      // give the copies in flight a bounded time to land before the CTA's shared memory is released
+      for (int q = max(0, n_stream - kRing); q < n_stream; ++q)
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->full[q % kRing]), (q / kRing) & 1); ++i) {}
+      if (issued_item > 0)
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->fixed_full), (issued_item - 1) & 1); ++i) {}
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(kTile, kTile);
+      int n_item = 0, n_stream = 0, cnt[2] = {0, 0};
+      bool ok = true;
+      while (ok) {
+        const int slot = n_item & 1;
+        ok = mbar_wait(smem_u32(&aux->item_full[slot]), (n_item >> 1) & 1, abort_flag);
+        if (!ok) break;
+        int it[5];
+#pragma unroll
+        for (int i = 0; i < 5; ++i) it[i] = aux->item[slot][i];
+        mbar_arrive(smem_u32(&aux->item_empty[slot]));
+        if (it[0] < 0) break;
+        const Geo<kColsum> g(s, it);
+        ok = mbar_wait(smem_u32(&aux->fixed_full), n_item & 1, abort_flag);
+        for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
+          const int rs = n_stream % kRing;
+          ok = mbar_wait(smem_u32(&aux->full[rs]), (n_stream / kRing) & 1, abort_flag);
+          for (int hf = 0; ok && hf < 2; ++hf) {
+            if (!g.active(hf, i)) continue;
+            const int c = cnt[hf]++;
+            const int buf = 2 * hf + (c & 1);
+            ok = mbar_wait(smem_u32(&aux->acc_empty[buf]), ((c >> 1) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * kTile;
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+              const uint32_t off = (k >> 2) * SL::kBlockBytes + (k & 3) * 32;
+              umma_bf16(d_tmem, smem_desc_sw128(fixed_addr + hf * SL::kTileBytes + off),
+                        smem_desc_sw128(ring_addr + rs * SL::kTileBytes + off), idesc, k > 0);
+            }
+            umma_commit(smem_u32(&aux->acc_full[buf]));
+          }
+          if (!ok) break;
+          umma_commit(smem_u32(&aux->empty[rs]));
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&aux->fixed_empty));
+        ++n_item;
+      }
+      if (*abort_flag) {
+        // wait (bounded) until every MMA already issued has retired before TMEM and shared memory go away
+        umma_commit(smem_u32(&aux->drain));
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->drain), 0); ++i) {}
+      }
+    }
+  } else {
+    // ------------------------------ epilogue groups ------------------------------
+    const int gi = (warp - 2) >> 2;                // group = half * 2 + parity
+    const int hf = gi >> 1, par = gi & 1;
+    const int quarter = warp & 3;                  // TMEM lanes this warp may read
+    const int r = quarter * 32 + lane;             // row of the accumulator = TMEM lane = index inside the group
+    const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + gi * kTile;
+    const uint32_t acc_full = smem_u32(&aux->acc_full[gi]), acc_empty = smem_u32(&aux->acc_empty[gi]);
+    const float scale = a.scale_log2;
+    const float inf = __int_as_float(0x7F800000);
+    int n_item = 0, cnt = 0, n_gsync = 0, n_psync = 0;
+    bool ok = true;
+
+    // barrier among the 4 warps of the group / the 8 warps of the half; bounded like every other wait
+    auto group_sync = [&]() {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&aux->group_bar[gi]));
+      ok = mbar_wait(smem_u32(&aux->group_bar[gi]), n_gsync & 1, abort_flag) && ok;
+      ++n_gsync;
+    };
+    auto pair_sync = [&]() {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&aux->pair_bar[hf]));
+      ok = mbar_wait(smem_u32(&aux->pair_bar[hf]), n_psync & 1, abort_flag) && ok;
+      ++n_psync;
+    };
+    auto release = [&]() {                         // accumulator drained: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty);
+    };
+
+    while (true) {
+      const int slot = n_item & 1;
+      ok = mbar_wait(smem_u32(&aux->item_full[slot]), (n_item >> 1) & 1, abort_flag) && ok;
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      int it[5];
+#pragma unroll
+      for (int i = 0; i < 5; ++i) it[i] = aux->item[slot][i];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&aux->item_empty[slot]));
+      if (it[0] < 0) break;
+      const Geo<kColsum> g(s, it);
+      const int row = g.blk * kBlockRows + hf * kTile + r;          // token of this thread inside the sequence
+      const size_t out = ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0 + row;
+
+      if constexpr (kColsum) {
+        const float* lse_row = a.lse + ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0;
+        auto load_lse = [&](int i) {                // lse2 of this thread's query of streamed tile i (+inf past the end)
+          const int j = (g.first_stream + i) * kTile + r;
+          return (i < g.n_iter && j < g.L) ? __ldg(lse_row + j) * a.lse_mul : inf;
+        };
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        // this group's tiles of the item: every other active tile, starting where the running parity says
+        int first = g.causal ? hf : 0;
+        if (((cnt & 1) != par)) ++first;
+        float lse_next = load_lse(first);
+        int n_mine = 0;
+        for (int i = 0; i < g.n_iter && ok; ++i) {
+          if (!g.active(hf, i)) continue;
+          const int c = cnt++;
+          if ((c & 1) != par) continue;
+          float* lse_buf = aux->lse_sh[gi][n_mine & 1];
+          ++n_mine;
+          lse_buf[r] = lse_next;
+          lse_next = load_lse(i + 2);               // in flight while this tile is processed
+          group_sync();
+          ok = mbar_wait(acc_full, (c >> 1) & 1, abort_flag) && ok;
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          if (g.diag(hf, i))
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
+          else
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
+        }
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        float total = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+        float* part = aux->part[hf][n_item & 1][0];
+        if (par == 1) part[r] = total;
+        pair_sync();
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        if (par == 0 && row < g.L && (hf == 0 || g.half1)) {
+          total += part[r];
+          if (a.normalize) total = total / (float)g.L;
+          a.scores[out] = total;
+        }
+      } else {
+        float m = __int_as_float(0xFF800000), sum = 0.f;        // running max (log2 domain) and sum of this row
+        for (int i = 0; i < g.n_iter && ok; ++i) {
+          if (!g.active(hf, i)) continue;
+          const int c = cnt++;
+          if ((c & 1) != par) continue;
+          ok = mbar_wait(acc_full, (c >> 1) & 1, abort_flag) && ok;
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          // keys of this tile that count for this row: up to the diagonal (causal) and inside the sequence
+          const int n_valid = g.causal ? (g.diag(hf, i) ? r + 1 : kTile) : min(kTile, g.L - i * kTile);
+          if (__any_sync(0xFFFFFFFFu, n_valid < kTile))
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, n_valid - p * 16, m, sum); }, release);
+          else
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, 16, m, sum); }, release);
+        }
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        float* pm = aux->part[hf][n_item & 1][0];
+        float* ps = aux->part[hf][n_item & 1][1];
+        if (par == 1) { pm[r] = m; ps[r] = sum; }
+        pair_sync();
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        if (par == 0 && row < g.L && (hf == 0 || g.half1)) {       // merge the other group's (max, sum)
+          const float m1 = pm[r], sum1 = ps[r];
+          const float big = fmaxf(m, m1);
+          const float tot = (sum > 0.f ? sum * ex2(m - big) : 0.f) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
+          const float lse2 = big + log2f(tot);
+          a.lse2_out[out] = lse2;
+          if (a.lse_nat_out) a.lse_nat_out[out] = lse2 * 0.69314718055994530942f;
+        }
+      }
+      ++n_item;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (tid == 0 && !dead && *abort_flag) report(a.status, KVCRUSH_DEV_TIMEOUT, kColsum ? KID_SCORE_COLSUM : KID_SCORE_LSE, blockIdx.x, 0);
+}
+
+template <int D, bool kColsum>
+int launch_persist(const CUtensorMap& mq, const CUtensorMap& mk, const PersistArgs& a, int n_sms, cudaStream_t stream) {
+  auto kern = score_persist_kernel<D, kColsum>;
+  constexpr int smem = PSmem<D>::kTotal;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return KVCRUSH_ERR_CUDA;
+  const int blocks = a.total_items < n_sms ? a.total_items : n_sms;
+  kern<<<(unsigned)blocks, kThreads, smem, stream>>>(mq, mk, a);
+  return check_launch();
+}
+
+}  // namespace
+
+size_t score_persist_counter_bytes() { return 256; }
+
+int launch_score_tensor_persistent(const Shape& s, const int32_t* cu_host, const TensorView& Q, const TensorView& K,
+                                   float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws,
+                                   int* counters, float* scores, float* lse_out, int normalize, int32_t* status,
+                                   cudaStream_t stream) {
+  static_assert(sizeof(PAux) <= 10240, "aux block too large");
+  if (!(scale_log2 > 0.f)) return KVCRUSH_ERR_UNSUPPORTED;
+  CUtensorMap mq, mk;
+  if (!make_map(&mq, Q, s.D, s.T, s.Hq, s.n_layers) || !make_map(&mk, K, s.D, s.T, s.Hkv, s.n_layers))
+    return KVCRUSH_ERR_CUDA;
+  int dev = 0, n_sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sms < 1)
+    return KVCRUSH_ERR_CUDA;
+  PersistArgs a{};
+  a.s = s; a.scale_log2 = scale_log2; a.normalize = normalize; a.status = status; a.scores = scores;
+  a.max_blocks = (s.max_seqlen + kBlockRows - 1) / kBlockRows;
+  long long items = 0;
+  for (int i = 0; i < s.n_seqs; ++i) items += (cu_host[i + 1] - cu_host[i] + kBlockRows - 1) / kBlockRows;
+  if (items == 0) return KVCRUSH_OK;
+  const long long total = items * s.n_layers * s.Hq;
+  if (total > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
+  a.n_items = (int)items;
+  a.total_items = (int)total;
+  if (cudaMemsetAsync(counters, 0, 2 * sizeof(int), stream) != cudaSuccess) return KVCRUSH_ERR_CUDA;
+  int rc;
+  if (!lse_in) {
+    a.lse2_out = lse2_ws; a.lse_nat_out = lse_out; a.counter = counters;
+    rc = s.D == 128 ? launch_persist<128, false>(mq, mk, a, n_sms, stream) : launch_persist<64, false>(mq, mk, a, n_sms, stream);
+    if (rc != KVCRUSH_OK) return rc;
+    a.lse = lse2_ws; a.lse_mul = 1.f;
+  } else {
+    a.lse = lse_in; a.lse_mul = lse_in_mul;
+  }
+  a.counter = counters + 1;
+  return s.D == 128 ? launch_persist<128, true>(mq, mk, a, n_sms, stream) : launch_persist<64, true>(mq, mk, a, n_sms, stream);
+}
+
+}  // namespace kvc

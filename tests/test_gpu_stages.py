@@ -178,7 +178,7 @@ def _score_case(B, w, impl, n_layers=None):
         np.testing.assert_allclose(gl[i], ol, rtol=0, atol=2e-4)
     # supplying the row log-sum-exp skips the first sweep and gives the same scores
     scores2 = torch.empty_like(scores)
-    B.kvcrush_score(prob, dq, dk, scores2, lse_in=lse, impl=impl, workspace=None, status=status)
+    B.kvcrush_score(prob, dq, dk, scores2, lse_in=lse, impl=impl, workspace=ws, status=status)
     torch.cuda.synchronize()
     np.testing.assert_allclose(scores2.cpu().numpy(), g, rtol=1e-4, atol=1e-6)
     # normalize = the paper's 1/S
