@@ -213,16 +213,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int gtid = r;                            // index inside the group (0..127)
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const float scale = a.scale_log2;
+    const f32x2 scale2 = splat2(scale);
     bool ok = true;
 
     if constexpr (kColsum) {
       const float* lse_row = a.lse + ((size_t)layer * s.Hq + h) * s.T + t0;
-      const float inf = __int_as_float(0x7F800000);
-      auto load_lse = [&](int it) {                 // lse2 of this thread's query of streamed tile `it` (+inf past the end)
+      const float ninf = __int_as_float(0xFF800000);
+      auto load_lse = [&](int it) {                 // minus lse2 of this thread's query of streamed tile `it` (-inf past the end)
         const int j = (first_stream + it) * kTile + gtid;
-        return (it < n_iter && j < L) ? __ldg(lse_row + j) * a.lse_mul : inf;
+        return (it < n_iter && j < L) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
       };
-      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      f32x2 acc[2] = {0ull, 0ull};
       float lse_next = load_lse(g);
       int n_mine = 0;
       for (int it = g; it < n_iter; it += kGroups, ++n_mine) {
@@ -244,11 +245,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         };
         const uint32_t t_acc = t_lane + b * kTile;
         if (s.causal && it == 0)
-          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
+          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
         else
-          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
+          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
       }
-      float total = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+      float total = sum4(acc);
       if constexpr (kGroups > 1) {
         if (g > 0) aux->part[g][0][r] = total;
         named_bar_sync(1 + kGroups, kGroups * kEpiThreads);
@@ -263,7 +264,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
       }
     } else {
-      float m = __int_as_float(0xFF800000), sum = 0.f;        // running max (log2 domain) and sum of this row
+      float m = __int_as_float(0xFF800000);                   // running max (log2 domain) of this row
+      f32x2 sum2[2] = {0ull, 0ull};                           // packed partial sums of 2^(x - m)
       for (int it = g; it < n_iter; it += kGroups) {
         const int b = it % kBufs;
         ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it / kBufs) & 1, abort_flag);
@@ -279,10 +281,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // keys of this tile that count for this row: up to the diagonal (causal) and inside the sequence
         const int n_valid = s.causal ? (it == my_tile ? r + 1 : kTile) : min(kTile, L - it * kTile);
         if (__any_sync(0xFFFFFFFFu, n_valid < kTile))
-          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, n_valid - p * 16, m, sum); }, release);
+          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, scale2, n_valid - p * 16, m, sum2); }, release);
         else
-          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, 16, m, sum); }, release);
+          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, scale2, 16, m, sum2); }, release);
       }
+      float sum = sum4(sum2);
       if constexpr (kGroups > 1) {
         if (g > 0) { aux->part[g][0][r] = m; aux->part[g][1][r] = sum; }
         named_bar_sync(1 + kGroups, kGroups * kEpiThreads);

@@ -277,7 +277,8 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + gi * kTile;
     const uint32_t acc_full = smem_u32(&aux->acc_full[gi]), acc_empty = smem_u32(&aux->acc_empty[gi]);
     const float scale = a.scale_log2;
-    const float inf = __int_as_float(0x7F800000);
+    const f32x2 scale2 = splat2(scale);
+    const float ninf = __int_as_float(0xFF800000);
     int n_item = 0, cnt = 0, n_gsync = 0, n_psync = 0;
     bool ok = true;
 
@@ -317,11 +318,11 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
       if constexpr (kColsum) {
         const float* lse_row = a.lse + ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0;
-        auto load_lse = [&](int i) {                // lse2 of this thread's query of streamed tile i (+inf past the end)
+        auto load_lse = [&](int i) {                // minus lse2 of this thread's query of streamed tile i (-inf past the end)
           const int j = (g.first_stream + i) * kTile + r;
-          return (i < g.n_iter && j < g.L) ? __ldg(lse_row + j) * a.lse_mul : inf;
+          return (i < g.n_iter && j < g.L) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
         };
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        f32x2 acc[2] = {0ull, 0ull};
         // this group's tiles of the item: every other active tile, starting where the running parity says
         int first = g.causal ? hf : 0;
         if (((cnt & 1) != par)) ++first;
@@ -341,13 +342,13 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           if (!ok) break;
           tc_fence_after();
           if (g.diag(hf, i))
-            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
           else
-            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale, r, p * 16, acc); }, release);
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
         }
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
-        float total = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+        float total = sum4(acc);
         float* part = aux->part[hf][n_item & 1][0];
         if (par == 1) part[r] = total;
         pair_sync();
@@ -359,7 +360,8 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           a.scores[out] = total;
         }
       } else {
-        float m = __int_as_float(0xFF800000), sum = 0.f;        // running max (log2 domain) and sum of this row
+        float m = __int_as_float(0xFF800000);                   // running max (log2 domain) of this row
+        f32x2 sum2[2] = {0ull, 0ull};                           // packed partial sums of 2^(x - m)
         for (int i = 0; i < g.n_iter && ok; ++i) {
           if (!g.active(hf, i)) continue;
           const int c = cnt++;
@@ -371,12 +373,13 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // keys of this tile that count for this row: up to the diagonal (causal) and inside the sequence
           const int n_valid = g.causal ? (g.diag(hf, i) ? r + 1 : kTile) : min(kTile, g.L - i * kTile);
           if (__any_sync(0xFFFFFFFFu, n_valid < kTile))
-            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, n_valid - p * 16, m, sum); }, release);
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, scale2, n_valid - p * 16, m, sum2); }, release);
           else
-            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, 16, m, sum); }, release);
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, scale2, 16, m, sum2); }, release);
         }
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
+        const float sum = sum4(sum2);
         float* pm = aux->part[hf][n_item & 1][0];
         float* ps = aux->part[hf][n_item & 1][1];
         if (par == 1) { pm[r] = m; ps[r] = sum; }

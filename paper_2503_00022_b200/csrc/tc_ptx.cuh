@@ -88,29 +88,72 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// 2^x on the FMA pipe for x <= ~0 (any magnitude): round-to-nearest split x = n + f, f in [-0.5, 0.5],
-// cubic minimax polynomial for 2^f (relative error 7.5e-5), exponent bits of n added to the result.
-// The special-function unit delivers 16 ex2 per clock per SM and is the busiest unit of both sweeps;
-// sending a fixed share of the exponentials down this path takes load off it.
-__device__ __forceinline__ float exp2_poly(float x) {
-  x = fmaxf(x, -125.f);                              // keeps the result a normal number (also maps -inf)
-  const float t = x + 12582912.f;                    // 1.5 * 2^23: the integer part lands in the low mantissa bits
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(f, 0.0551716648f, 0.2426111251f);
-  p = fmaf(p, f, 0.6932609677f);
-  p = fmaf(p, f, 0.9999280572f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+// ---- packed fp32x2 arithmetic (two floats in one 64-bit register, one instruction for both) ---------
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(uint32_t lo, uint32_t hi) {
+  f32x2 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+__device__ __forceinline__ f32x2 pack2f(float lo, float hi) { return pack2(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ f32x2 splat2(float x) { return pack2f(x, x); }
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a);
+  hi = __uint_as_float(b);
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
 }
 
-#ifndef KVC_POLY_PER8
-#define KVC_POLY_PER8 2                              // of every 8 exponentials, this many use exp2_poly
-#endif
-__host__ __device__ constexpr bool poly_slot(int i) {
-  return ((i % 8 + 1) * KVC_POLY_PER8) / 8 > ((i % 8) * KVC_POLY_PER8) / 8;
+// 2^x for a pair on the special-function unit.
+__device__ __forceinline__ f32x2 exp2_sfu2(f32x2 x) {
+  float a, b;
+  unpack2(x, a, b);
+  return pack2f(ex2(a), ex2(b));
 }
-template <int I>
-__device__ __forceinline__ float exp2_mix(float x) {
-  if constexpr (poly_slot(I)) return exp2_poly(x); else return ex2(x);
+// 2^x for a pair on the FMA pipe, x <= ~0 (any magnitude): round-to-nearest split x = n + f, f in [-0.5, 0.5],
+// cubic minimax polynomial for 2^f (relative error 7.5e-5), exponent bits of n added to the result.
+// The special-function unit delivers 16 ex2 per clock per SM and is the busiest unit of both sweeps; a
+// share of the exponentials can go down this path instead, at 6 packed + 6 scalar instructions a pair.
+__device__ __forceinline__ f32x2 exp2_poly2(f32x2 x) {
+  float x0, x1;
+  unpack2(x, x0, x1);
+  x = pack2f(fmaxf(x0, -125.f), fmaxf(x1, -125.f));           // keeps the result a normal number (also maps -inf)
+  const f32x2 t = add2(x, splat2(12582912.f));                // 1.5 * 2^23: the integer part lands in the low mantissa bits
+  const f32x2 n = add2(t, splat2(-12582912.f));
+  const f32x2 f = fma2(n, splat2(-1.f), x);
+  f32x2 p = fma2(f, splat2(0.0551716648f), splat2(0.2426111251f));
+  p = fma2(p, f, splat2(0.6932609677f));
+  p = fma2(p, f, splat2(0.9999280572f));
+  float p0, p1, t0, t1;
+  unpack2(p, p0, p1);
+  unpack2(t, t0, t1);
+  return pack2(__float_as_uint(p0) + (__float_as_uint(t0) << 23), __float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
+
+#ifndef KVC_POLY_PAIRS_PER4
+#define KVC_POLY_PAIRS_PER4 1                        // of every 4 pairs of exponentials, this many use exp2_poly2
+#endif
+__host__ __device__ constexpr bool poly_pair(int j) {
+  return ((j % 4 + 1) * KVC_POLY_PAIRS_PER4) / 4 > ((j % 4) * KVC_POLY_PAIRS_PER4) / 4;
+}
+template <int J>
+__device__ __forceinline__ f32x2 exp2_mix2(f32x2 x) {
+  if constexpr (poly_pair(J)) return exp2_poly2(x); else return exp2_sfu2(x);
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -158,62 +201,73 @@ __device__ __forceinline__ void sweep_tile(uint32_t taddr, Piece&& piece, Releas
 }
 
 // ---- sweep 2: 16 columns (queries) of this thread's key row -------------------------------------
-template <bool kDiag>
-__device__ __forceinline__ void colsum_piece(const uint32_t (&v)[16], const float* lse16, float scale, int r, int c0,
-                                             float (&acc)[4]) {
-  const float4* l4 = reinterpret_cast<const float4*>(lse16);
-#pragma unroll
-  for (int c4 = 0; c4 < 4; ++c4) {
-    const float4 l = l4[c4];
-    float e0, e1, e2, e3;
-    if (c4 == 0) {
-      e0 = exp2_mix<0>(fmaf(__uint_as_float(v[0]), scale, -l.x)); e1 = exp2_mix<1>(fmaf(__uint_as_float(v[1]), scale, -l.y));
-      e2 = exp2_mix<2>(fmaf(__uint_as_float(v[2]), scale, -l.z)); e3 = exp2_mix<3>(fmaf(__uint_as_float(v[3]), scale, -l.w));
-    } else if (c4 == 1) {
-      e0 = exp2_mix<4>(fmaf(__uint_as_float(v[4]), scale, -l.x)); e1 = exp2_mix<5>(fmaf(__uint_as_float(v[5]), scale, -l.y));
-      e2 = exp2_mix<6>(fmaf(__uint_as_float(v[6]), scale, -l.z)); e3 = exp2_mix<7>(fmaf(__uint_as_float(v[7]), scale, -l.w));
-    } else if (c4 == 2) {
-      e0 = exp2_mix<0>(fmaf(__uint_as_float(v[8]), scale, -l.x)); e1 = exp2_mix<1>(fmaf(__uint_as_float(v[9]), scale, -l.y));
-      e2 = exp2_mix<2>(fmaf(__uint_as_float(v[10]), scale, -l.z)); e3 = exp2_mix<3>(fmaf(__uint_as_float(v[11]), scale, -l.w));
-    } else {
-      e0 = exp2_mix<4>(fmaf(__uint_as_float(v[12]), scale, -l.x)); e1 = exp2_mix<5>(fmaf(__uint_as_float(v[13]), scale, -l.y));
-      e2 = exp2_mix<6>(fmaf(__uint_as_float(v[14]), scale, -l.z)); e3 = exp2_mix<7>(fmaf(__uint_as_float(v[15]), scale, -l.w));
-    }
-    if constexpr (kDiag) {                          // causal: the query (column) must not precede the key (row)
-      const int c = c0 + 4 * c4;
-      e0 = c + 0 >= r ? e0 : 0.f; e1 = c + 1 >= r ? e1 : 0.f;
-      e2 = c + 2 >= r ? e2 : 0.f; e3 = c + 3 >= r ? e3 : 0.f;
-    }
-    acc[0] += e0; acc[1] += e1; acc[2] += e2; acc[3] += e3;
+// nlse16: MINUS the log2-domain row log-sum-exp of the 16 queries (-inf past the end of the sequence).
+template <int J, bool kDiag>
+__device__ __forceinline__ f32x2 colsum_pair(uint32_t v0, uint32_t v1, float nl0, float nl1, f32x2 scale2, int r, int c) {
+  f32x2 e = exp2_mix2<J>(fma2(pack2(v0, v1), scale2, pack2f(nl0, nl1)));
+  if constexpr (kDiag) {                            // causal: the query (column) must not precede the key (row)
+    float e0, e1;
+    unpack2(e, e0, e1);
+    e = pack2f(c >= r ? e0 : 0.f, c + 1 >= r ? e1 : 0.f);
   }
+  return e;
+}
+template <bool kDiag>
+__device__ __forceinline__ void colsum_piece(const uint32_t (&v)[16], const float* nlse16, f32x2 scale2, int r, int c0,
+                                             f32x2 (&acc)[2]) {
+  const float4* l4 = reinterpret_cast<const float4*>(nlse16);
+  const float4 la = l4[0], lb = l4[1], lc = l4[2], ld = l4[3];
+  acc[0] = add2(acc[0], colsum_pair<0, kDiag>(v[0], v[1], la.x, la.y, scale2, r, c0 + 0));
+  acc[1] = add2(acc[1], colsum_pair<1, kDiag>(v[2], v[3], la.z, la.w, scale2, r, c0 + 2));
+  acc[0] = add2(acc[0], colsum_pair<2, kDiag>(v[4], v[5], lb.x, lb.y, scale2, r, c0 + 4));
+  acc[1] = add2(acc[1], colsum_pair<3, kDiag>(v[6], v[7], lb.z, lb.w, scale2, r, c0 + 6));
+  acc[0] = add2(acc[0], colsum_pair<0, kDiag>(v[8], v[9], lc.x, lc.y, scale2, r, c0 + 8));
+  acc[1] = add2(acc[1], colsum_pair<1, kDiag>(v[10], v[11], lc.z, lc.w, scale2, r, c0 + 10));
+  acc[0] = add2(acc[0], colsum_pair<2, kDiag>(v[12], v[13], ld.x, ld.y, scale2, r, c0 + 12));
+  acc[1] = add2(acc[1], colsum_pair<3, kDiag>(v[14], v[15], ld.z, ld.w, scale2, r, c0 + 14));
 }
 
 // ---- sweep 1: 16 columns (keys) of this thread's query row; online max / sum in the log2 domain ----
+// m: running maximum; sum2: two packed partial sums of 2^(x - m) (four floats to add up at the end).
 template <bool kMasked>
-__device__ __forceinline__ void lse_piece(const uint32_t (&v)[16], float scale, int c_lim, float& m, float& sum) {
-  float x[16];
+__device__ __forceinline__ void lse_piece(const uint32_t (&v)[16], float scale, f32x2 scale2, int c_lim, float& m,
+                                          f32x2 (&sum2)[2]) {
+  uint32_t x[16];
 #pragma unroll
-  for (int c = 0; c < 16; ++c) x[c] = __uint_as_float(v[c]);
+  for (int c = 0; c < 16; ++c) x[c] = v[c];
   if constexpr (kMasked) {
     if (c_lim <= 0) return;                         // nothing of this piece belongs to the row
 #pragma unroll
-    for (int c = 0; c < 16; ++c) x[c] = c < c_lim ? x[c] : __int_as_float(0xFF800000);
+    for (int c = 0; c < 16; ++c) x[c] = c < c_lim ? x[c] : 0xFF800000u;
   }
-  const float m0 = max3(x[0], x[1], x[2]), m1 = max3(x[3], x[4], x[5]), m2 = max3(x[6], x[7], x[8]);
-  const float m3 = max3(x[9], x[10], x[11]), m4 = max3(x[12], x[13], x[14]);
-  const float cmax = fmaxf(max3(m0, m1, m2), max3(m3, m4, x[15]));
+#define KVC_F(i) __uint_as_float(x[i])
+  const float m0 = max3(KVC_F(0), KVC_F(1), KVC_F(2)), m1 = max3(KVC_F(3), KVC_F(4), KVC_F(5));
+  const float m2 = max3(KVC_F(6), KVC_F(7), KVC_F(8)), m3 = max3(KVC_F(9), KVC_F(10), KVC_F(11));
+  const float m4 = max3(KVC_F(12), KVC_F(13), KVC_F(14));
+  const float cmax = fmaxf(max3(m0, m1, m2), max3(m3, m4, KVC_F(15)));
+#undef KVC_F
   const float m_new = fmaxf(m, cmax * scale);
-  if (m_new > m) { sum *= ex2(m - m_new); m = m_new; }
-  float s0, s1, s2, s3;
-  s0 = exp2_mix<0>(fmaf(x[0], scale, -m)); s1 = exp2_mix<1>(fmaf(x[1], scale, -m));
-  s2 = exp2_mix<2>(fmaf(x[2], scale, -m)); s3 = exp2_mix<3>(fmaf(x[3], scale, -m));
-  s0 += exp2_mix<4>(fmaf(x[4], scale, -m)); s1 += exp2_mix<5>(fmaf(x[5], scale, -m));
-  s2 += exp2_mix<6>(fmaf(x[6], scale, -m)); s3 += exp2_mix<7>(fmaf(x[7], scale, -m));
-  s0 += exp2_mix<0>(fmaf(x[8], scale, -m)); s1 += exp2_mix<1>(fmaf(x[9], scale, -m));
-  s2 += exp2_mix<2>(fmaf(x[10], scale, -m)); s3 += exp2_mix<3>(fmaf(x[11], scale, -m));
-  s0 += exp2_mix<4>(fmaf(x[12], scale, -m)); s1 += exp2_mix<5>(fmaf(x[13], scale, -m));
-  s2 += exp2_mix<6>(fmaf(x[14], scale, -m)); s3 += exp2_mix<7>(fmaf(x[15], scale, -m));
-  sum += (s0 + s1) + (s2 + s3);
+  if (m_new > m) {
+    const f32x2 corr = splat2(ex2(m - m_new));
+    sum2[0] = mul2(sum2[0], corr);
+    sum2[1] = mul2(sum2[1], corr);
+    m = m_new;
+  }
+  const f32x2 nm = splat2(-m);
+  sum2[0] = add2(sum2[0], exp2_mix2<0>(fma2(pack2(x[0], x[1]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<1>(fma2(pack2(x[2], x[3]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<2>(fma2(pack2(x[4], x[5]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<3>(fma2(pack2(x[6], x[7]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<0>(fma2(pack2(x[8], x[9]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<1>(fma2(pack2(x[10], x[11]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<2>(fma2(pack2(x[12], x[13]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<3>(fma2(pack2(x[14], x[15]), scale2, nm)));
+}
+__device__ __forceinline__ float sum4(const f32x2 (&s)[2]) {
+  float a, b, c, d;
+  unpack2(s[0], a, b);
+  unpack2(s[1], c, d);
+  return (a + b) + (c + d);
 }
 
 // Shared-memory matrix descriptor of a K-major tile stored as 128-byte rows with the 128B swizzle
