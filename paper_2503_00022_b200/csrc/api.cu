@@ -48,7 +48,7 @@ int make_view(const kvcrush_tensor_t* t, int head_dim, TensorView* v) {
 
 size_t score_lse_bytes(const Shape& s) { return round_up((size_t)s.n_layers * s.Hq * s.T * sizeof(float)); }
 // row log-sum-exp of every query + the work counters of the persistent tensor-core kernels
-size_t score_ws(const Shape& s) { return score_lse_bytes(s) + round_up(score_persist_counter_bytes()); }
+size_t score_ws(const Shape& s) { return score_lse_bytes(s) + round_up(score_tensor_counter_bytes()); }
 size_t signature_ws(const Shape& s) { return round_up((size_t)s.n_layers * s.n_seqs * s.Hq * sizeof(float)); }
 
 }  // namespace
@@ -100,14 +100,8 @@ int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, c
   if (impl == KVCRUSH_SCORE_SIMT || !tensor_ok)
     return launch_score_simt(s, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, scores_dev, lse_out_dev, normalize,
                              status_dev, st);
-#ifndef KVC_TENSOR_PERSISTENT
-  (void)counters;
-  return launch_score_tensor(s, problem->cu_seqlens_host, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, scores_dev,
-                             lse_out_dev, normalize, status_dev, st);
-#else
-  return launch_score_tensor_persistent(s, problem->cu_seqlens_host, q, k, scale_log2, lse_in_dev, log2e, lse2_ws,
-                                        counters, scores_dev, lse_out_dev, normalize, status_dev, st);
-#endif
+  return launch_score_tensor(s, problem->cu_seqlens_host, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, counters,
+                             scores_dev, lse_out_dev, normalize, status_dev, st);
 }
 
 int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev, const int32_t* sig_keep_dev,

@@ -53,16 +53,11 @@ int launch_score_simt(const Shape& s, const TensorView& Q, const TensorView& K, 
                       const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores, float* lse_out,
                       int normalize, int32_t* status, cudaStream_t stream);
 bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorView& K);
+// `counters`: two ints of caller scratch (work counters of the two persistent sweeps).
+size_t score_tensor_counter_bytes();
 int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView& Q, const TensorView& K,
-                        float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores,
-                        float* lse_out, int normalize, int32_t* status, cudaStream_t stream);
-
-// Persistent variant (one CTA per SM, 256-row work items); `counters` = two ints of caller scratch.
-size_t score_persist_counter_bytes();
-int launch_score_tensor_persistent(const Shape& s, const int32_t* cu_host, const TensorView& Q, const TensorView& K,
-                                   float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws,
-                                   int* counters, float* scores, float* lse_out, int normalize, int32_t* status,
-                                   cudaStream_t stream);
+                        float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws, int* counters,
+                        float* scores, float* lse_out, int normalize, int32_t* status, cudaStream_t stream);
 
 int launch_signature(const Shape& s, const float* scores, const int32_t* sig_keep, const float* theta_in,
                      uint32_t* sigs, float* theta, cudaStream_t stream);

@@ -1,27 +1,32 @@
 // Stage 1 on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16 Q/K, head_dim 64 or 128.
 //
-// Attention column sums (Algorithm 1 of the paper: A_h = softmax(Q_h K_h^T / sqrt(d_k)), then the
-// per-token sum of A_h over the queries) without ever storing the S x S matrix: two sweeps that
-// both recompute 128 x 128 logit tiles.
+// Attention column sums (Algorithm 1 of the paper: A_h = softmax(Q_h K_h^T / sqrt(d_k)), then the per-token
+// sum of A_h over the queries) without ever storing the S x S matrix: two sweeps that both recompute
+// 128 x 128 logit tiles.
 //
-//   sweep 1 (kColsum = false)  one CTA per (layer, head, sequence, 128-query tile): S = Q_tile K^T,
-//                              TMEM lane = query row, so each epilogue thread owns one row and keeps
-//                              its running (max, sum) in registers  ->  lse2(j) = log2 sum_t 2^(s2(j,t))
-//   sweep 2 (kColsum = true)   one CTA per (layer, head, sequence, 128-key tile): S^T = K_tile Q^T,
-//                              TMEM lane = key, so each epilogue thread owns one key column and adds
-//                              2^(s2 - lse2(j)) = A(j, t) over all query tiles in a register.
+//   sweep 1 (kColsum = false)  S = Q_block K^T: TMEM lane = query row, so each epilogue thread owns one row
+//                              and keeps its running (max, sum) in registers -> lse2(j) = log2 sum_t 2^(s2(j,t))
+//   sweep 2 (kColsum = true)   S^T = K_block Q^T: TMEM lane = key, so each epilogue thread owns one key column
+//                              and adds 2^(s2 - lse2(j)) = A(j, t) over all query tiles in registers.
 //                              No shuffles or atomics: one deterministic store per key.
 //   s2 = q.k * softmax_scale * log2(e).
 //
-// CTA = 10 warps: warp 0 issues TMA loads (one lane), warp 1 allocates TMEM and issues tcgen05.mma
-// (one lane), warps 2..9 are two epilogue groups of 128 threads that take alternate tiles, each
-// reading its own 128-column TMEM accumulator, so the MMA of tile i+1 overlaps the exponentials of
-// tile i.  The stationary operand stays in shared memory for the CTA's life; the streamed operand
-// runs through a ring of 128B-swizzled stages.  Two CTAs fit one SM (96 KB shared memory, 256 TMEM
-// columns each).  CTAs are ordered heaviest-first (causal rows/columns have 1..n tiles).
-// Every barrier wait is bounded; on expiry the CTA flags status, drains its copies and exits.
+// On this part the sweeps run against the board's power limit, so the work decomposition is built to
+// spend little energy per logit tile:
+//
+//   * one CTA per SM lives for the whole launch and pulls work items from an atomic counter, so TMEM
+//     allocation, barrier set-up and pipeline fill are paid once per SM instead of once per item;
+//   * an item is a 256-row block of the stationary operand (two 128-row halves).  Every streamed
+//     128-row tile is multiplied with both halves, which halves the L2 -> shared-memory traffic per logit;
+//   * TMEM holds four 128-column accumulators, two per half, so the tensor core fills one buffer of a half
+//     while an epilogue group drains the other.
+//
+// Roles: warp 0 fetches + decodes items and issues TMA loads; warp 1 (one lane) issues tcgen05.mma;
+// warps 2..17 are four epilogue groups (half x buffer parity) of 128 threads, thread = TMEM lane = one
+// query row (sweep 1) or one key column (sweep 2).  All synchronisation is by mbarriers with bounded
+// waits: a role that gives up sets the CTA's abort flag, every other wait then ends, the CTA reports
+// through the status word, drains its copies, frees TMEM and returns.
 #include <cuda.h>
-#include <cuda_bf16.h>
 
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -30,102 +35,120 @@ namespace kvc {
 
 namespace {
 
-constexpr int kTile = 128;               // rows of both operands per tile
-#ifndef KVC_EPI_GROUPS
-#define KVC_EPI_GROUPS 2
-#endif
-constexpr int kGroups = KVC_EPI_GROUPS;  // epilogue groups of 128 threads; tile i goes to group i % kGroups
-constexpr int kEpiThreads = 128;         // per epilogue group
-constexpr int kThreads = 64 + kGroups * kEpiThreads;
-constexpr int kBufs = kGroups < 2 ? 2 : kGroups;         // 128-column fp32 accumulators in TMEM; tile i uses buffer i % kBufs
-constexpr uint32_t kTmemCols = kBufs * 128;
-constexpr int kCtasPerSm = kGroups > 2 ? 1 : 2;
-#ifndef KVC_STAGES
-#define KVC_STAGES (kGroups > 2 ? 5 : 2)
-#endif
-constexpr int kStages = KVC_STAGES;      // ring depth of the streamed operand
-
 using namespace tc;
 
-struct ScoreArgs {
+constexpr int kTile = 128;
+constexpr int kBlockRows = 2 * kTile;        // stationary rows per work item
+constexpr int kEpiWarps = 16;
+constexpr int kThreads = 64 + kEpiWarps * 32;
+constexpr int kRing = 4;                     // streamed tiles in flight
+constexpr uint32_t kTmemCols = 512;          // 4 accumulators x 128 fp32 columns
+
+struct PersistArgs {
   Shape s;
   float scale_log2;
-  const float* lse;       // sweep 2: row log-sum-exp; value * lse_mul is in the log2 domain
+  const float* lse;        // sweep 2: row log-sum-exp; value * lse_mul is in the log2 domain
   float lse_mul;
-  float* lse2_out;        // sweep 1: log2-domain output [n_layers][Hq][T]
-  float* lse_nat_out;     // sweep 1: optional natural-log copy
-  float* scores;          // sweep 2 output
+  float* lse2_out;         // sweep 1 output (log2 domain), [n_layers][Hq][T]
+  float* lse_nat_out;      // sweep 1: optional natural-log copy
+  float* scores;           // sweep 2 output
   int normalize;
-  int max_tiles;          // ceil(max_seqlen / 128)
-  int n_items;            // number of (sequence, tile) pairs
+  int max_blocks;          // ceil(max_seqlen / 256)
+  int n_items;             // (sequence, 256-row block) pairs of one (layer, head)
+  int total_items;         // n_items * n_layers * Hq
+  int* counter;            // work counter, zero at launch
   int32_t* status;
 };
 
 template <int D>
-struct SmemLayout {
+struct PSmem {
   static constexpr int kTileBytes = kTile * D * 2;
-  static constexpr int kBlockBytes = kTile * 128;            // one 64-element k-block of a tile
-  static constexpr int kFixedOff = 0;
-  static constexpr int kRingOff = kTileBytes;
-  static constexpr int kAuxOff = kRingOff + kStages * kTileBytes;
-  static constexpr int kAuxBytes = 12288;
-  static constexpr int kTotal = kAuxOff + kAuxBytes + 1024;  // + slack to align the base to 1024
+  static constexpr int kBlockBytes = kTile * 128;
+  static constexpr int kFixedOff = 0;                            // two stationary halves
+  static constexpr int kRingOff = 2 * kTileBytes;
+  static constexpr int kAuxOff = kRingOff + kRing * kTileBytes;
+  static constexpr int kAuxBytes = 10240;
+  static constexpr int kTotal = kAuxOff + kAuxBytes + 1024;
 };
 
-struct Aux {                         // lives at kAuxOff
-  unsigned long long full[kStages];
-  unsigned long long empty[kStages];
-  unsigned long long fixed_full;
-  unsigned long long acc_full[kBufs];
-  unsigned long long acc_empty[kBufs];
+struct PAux {
+  unsigned long long full[kRing], empty[kRing];
+  unsigned long long fixed_full, fixed_empty;
+  unsigned long long acc_full[4], acc_empty[4];       // [half * 2 + parity]
+  unsigned long long item_full[2], item_empty[2];
+  unsigned long long pair_bar[2];                     // both groups of one half (8 warps)
+  unsigned long long group_bar[4];                    // one group (4 warps)
   unsigned long long drain;
   uint32_t tmem_base;
   int abort_flag;
-  int item[4];                       // seq, tile, n_tiles
-  alignas(16) float lse_sh[kGroups][2][kTile];   // [group][buffer][query in tile]   (sweep 2)
-  alignas(16) float part[kGroups][2][kTile];     // partials of groups 1.. handed to group 0
+  int item[2][8];                                     // layer, head, seq, block, n_tiles (layer < 0: no more work)
+  alignas(16) float lse_sh[4][2][kTile];              // [group][buffer][query of the streamed tile]
+  alignas(16) float part[2][2][2][kTile];             // [half][item parity][value][row]
+};
+
+// Geometry of one work item, derived identically by every role.
+template <bool kColsum>
+struct Geo {
+  int layer, h, hk, t0, L, blk, first_stream, n_iter;
+  bool causal, half1;
+  __device__ __forceinline__ Geo(const Shape& s, const int* it) {
+    layer = it[0]; h = it[1]; hk = h / s.G; blk = it[3];
+    const int seq = it[2], n_tiles = it[4];
+    t0 = __ldg(s.cu_seqlens + seq);
+    L = __ldg(s.cu_seqlens + seq + 1) - t0;
+    causal = s.causal != 0;
+    half1 = blk * kBlockRows + kTile < L;                               // does the second half hold any row
+    if (kColsum) {                                                      // stationary keys, streamed query tiles
+      first_stream = causal ? 2 * blk : 0;
+      n_iter = n_tiles - first_stream;
+    } else {                                                            // stationary queries, streamed key tiles
+      first_stream = 0;
+      n_iter = causal ? min(2 * blk + 2, n_tiles) : n_tiles;
+    }
+  }
+  // does streamed tile `it` contribute to half `hf` (causal: the half's own tile index is 2*blk + hf)
+  __device__ __forceinline__ bool active(int hf, int it) const {
+    if (hf == 1 && !half1) return false;
+    if (!causal) return true;
+    return kColsum ? it >= hf : it <= 2 * blk + hf;
+  }
+  __device__ __forceinline__ bool diag(int hf, int it) const {
+    return causal && (kColsum ? it == hf : it == 2 * blk + hf);
+  }
 };
 
 template <int D, bool kColsum>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
-score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                const ScoreArgs a) {
-  using SL = SmemLayout<D>;
+__global__ void __launch_bounds__(kThreads, 1)
+score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                     const PersistArgs a) {
+  using SL = PSmem<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  Aux* aux = reinterpret_cast<Aux*>(smem + SL::kAuxOff);
+  PAux* aux = reinterpret_cast<PAux*>(smem + SL::kAuxOff);
   volatile int* abort_flag = &aux->abort_flag;
   const uint32_t fixed_addr = smem_u32(smem + SL::kFixedOff);
   const uint32_t ring_addr = smem_u32(smem + SL::kRingOff);
-
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Shape& s = a.s;
-#ifdef KVC_RANK_MAJOR
-  const int n_lh = s.n_layers * s.Hq;
-#endif
-  // Block order: all tile-rows of one (layer, head) are adjacent, heaviest first, so the CTAs that run
-  // at the same time stream the same few heads' Q/K and those stay in L2.
-#ifdef KVC_RANK_MAJOR
-  const int lh = blockIdx.x % n_lh;
-  const int rank = blockIdx.x / n_lh;
-#else
-  const int lh = blockIdx.x / a.n_items;
-  const int rank = blockIdx.x - lh * a.n_items;
-#endif
-  const int layer = lh / s.Hq, h = lh - layer * s.Hq;
-  const int hk = h / s.G;
 
   if (warp == 0) {
-    int seq, tile, nt;
-    decode_item(s.cu_seqlens, s.n_seqs, a.max_tiles, rank, !kColsum, lane, seq, tile, nt);
     if (lane == 0) {
-      aux->item[0] = seq; aux->item[1] = tile; aux->item[2] = nt;
-      // a launch that already failed somewhere is not worth finishing: later CTAs leave at once
+      // a launch that already failed somewhere is not worth finishing
       aux->abort_flag = *reinterpret_cast<volatile int32_t*>(a.status) != 0;
-      for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&aux->full[i]), 1); mbar_init(smem_u32(&aux->empty[i]), 1); }
+      for (int i = 0; i < kRing; ++i) { mbar_init(smem_u32(&aux->full[i]), 1); mbar_init(smem_u32(&aux->empty[i]), 1); }
       mbar_init(smem_u32(&aux->fixed_full), 1);
+      mbar_init(smem_u32(&aux->fixed_empty), 1);
       mbar_init(smem_u32(&aux->drain), 1);
-      for (int i = 0; i < kBufs; ++i) { mbar_init(smem_u32(&aux->acc_full[i]), 1); mbar_init(smem_u32(&aux->acc_empty[i]), 4); }
+      for (int i = 0; i < 4; ++i) {
+        mbar_init(smem_u32(&aux->acc_full[i]), 1);
+        mbar_init(smem_u32(&aux->acc_empty[i]), 4);
+        mbar_init(smem_u32(&aux->group_bar[i]), 4);
+      }
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(smem_u32(&aux->item_full[i]), 1);
+        mbar_init(smem_u32(&aux->item_empty[i]), 1 + kEpiWarps);
+        mbar_init(smem_u32(&aux->pair_bar[i]), 8);
+      }
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -136,70 +159,122 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-
-  const int seq = aux->item[0], my_tile = aux->item[1], n_tiles = aux->item[2];
   const uint32_t tmem_base = aux->tmem_base;
-  const int t0 = __ldg(s.cu_seqlens + seq);
-  const int L = __ldg(s.cu_seqlens + seq + 1) - t0;
-  // tiles of the streamed operand swept by this CTA
-  const int first_stream = kColsum ? (s.causal ? my_tile : 0) : 0;
-  const int n_iter = s.causal ? (kColsum ? n_tiles - my_tile : my_tile + 1) : n_tiles;
-  // sweep 1: A = Q tile (stationary), B = K tiles.  sweep 2: A = K tile (stationary), B = Q tiles.
+  const bool dead = aux->abort_flag != 0;
+
   const CUtensorMap* map_fixed = kColsum ? &map_k : &map_q;
   const CUtensorMap* map_stream = kColsum ? &map_q : &map_k;
-  const int head_fixed = kColsum ? hk : h, head_stream = kColsum ? h : hk;
 
-  const bool dead = aux->abort_flag != 0;
   if (dead) {
     // nothing to do
   } else if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
-      mbar_expect_tx(smem_u32(&aux->fixed_full), SL::kTileBytes);
-#pragma unroll
-      for (int kb = 0; kb < D / 64; ++kb)
-        tma_load_4d(fixed_addr + kb * SL::kBlockBytes, map_fixed, smem_u32(&aux->fixed_full), kb * 64,
-                    t0 + my_tile * kTile, head_fixed, layer);
-      int issued = 0;
-      for (int it = 0; it < n_iter; ++it) {
-        const int st = it % kStages;
-        if (!mbar_wait(smem_u32(&aux->empty[st]), ((it / kStages) & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(smem_u32(&aux->full[st]), SL::kTileBytes);
-#pragma unroll
-        for (int kb = 0; kb < D / 64; ++kb)
-          tma_load_4d(ring_addr + st * SL::kTileBytes + kb * SL::kBlockBytes, map_stream, smem_u32(&aux->full[st]),
-                      kb * 64, t0 + (first_stream + it) * kTile, head_stream, layer);
-        issued = it + 1;
+    // ------------------------------ work fetch + TMA producer ------------------------------
+    int n_item = 0, n_stream = 0;
+    int issued_item = 0;              // lane 0: items whose stationary load was issued
+    bool alive = true;
+    while (alive) {
+      const int slot = n_item & 1;
+      int idx = 0;
+      bool ok = true;
+      if (lane == 0) {
+        ok = mbar_wait(smem_u32(&aux->item_empty[slot]), ((n_item >> 1) & 1) ^ 1, abort_flag);
+        if (ok) idx = atomicAdd(a.counter, 1);
       }
-      if (*abort_flag) {
-        // give the copies in flight a bounded time to land before the CTA's shared memory is released
-        for (int it = max(0, issued - kStages); it < issued; ++it)
-          for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->full[it % kStages]), (it / kStages) & 1); ++i) {}
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->fixed_full), 0); ++i) {}
+      ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+      idx = __shfl_sync(0xFFFFFFFFu, idx, 0);
+      if (!ok) break;
+      if (idx >= a.total_items) {
+        if (lane == 0) { aux->item[slot][0] = -1; mbar_arrive(smem_u32(&aux->item_full[slot])); }
+        break;
       }
+      const int lh = idx / a.n_items, rank = idx - lh * a.n_items;
+      int seq, blk, nblk;
+      decode_item(s.cu_seqlens, s.n_seqs, a.max_blocks, rank, !kColsum, lane, seq, blk, nblk, kBlockRows);
+      if (lane == 0) {
+        int* it = aux->item[slot];
+        it[0] = lh / s.Hq; it[1] = lh - it[0] * s.Hq; it[2] = seq; it[3] = blk;
+        it[4] = (__ldg(s.cu_seqlens + seq + 1) - __ldg(s.cu_seqlens + seq) + kTile - 1) / kTile;
+        mbar_arrive(smem_u32(&aux->item_full[slot]));
+        const Geo<kColsum> g(s, it);
+        const int head_fixed = kColsum ? g.hk : g.h, head_stream = kColsum ? g.h : g.hk;
+        // the stationary buffer is free once every MMA of the previous item has retired
+        ok = mbar_wait(smem_u32(&aux->fixed_empty), (n_item & 1) ^ 1, abort_flag);
+        if (ok) {
+          const int n_half = g.half1 ? 2 : 1;
+          mbar_expect_tx(smem_u32(&aux->fixed_full), n_half * SL::kTileBytes);
+          for (int hf = 0; hf < n_half; ++hf)
+#pragma unroll
+            for (int kb = 0; kb < D / 64; ++kb)
+              tma_load_4d(fixed_addr + hf * SL::kTileBytes + kb * SL::kBlockBytes, map_fixed, smem_u32(&aux->fixed_full),
+                          kb * 64, g.t0 + g.blk * kBlockRows + hf * kTile, head_fixed, g.layer);
+          issued_item = n_item + 1;
+          for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
+            const int rs = n_stream % kRing;
+            ok = mbar_wait(smem_u32(&aux->empty[rs]), ((n_stream / kRing) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(smem_u32(&aux->full[rs]), SL::kTileBytes);
+#pragma unroll
+            for (int kb = 0; kb < D / 64; ++kb)
+              tma_load_4d(ring_addr + rs * SL::kTileBytes + kb * SL::kBlockBytes, map_stream, smem_u32(&aux->full[rs]),
+                          kb * 64, g.t0 + (g.first_stream + i) * kTile, head_stream, g.layer);
+          }
+        }
+      }
+      alive = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+      n_stream = __shfl_sync(0xFFFFFFFFu, n_stream, 0);
+      ++n_item;
+    }
+    if (lane == 0 && *abort_flag) {
+      // give the copies in flight a bounded time to land before the CTA's shared memory is released
+      for (int q = max(0, n_stream - kRing); q < n_stream; ++q)
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->full[q % kRing]), (q / kRing) & 1); ++i) {}
+      if (issued_item > 0)
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->fixed_full), (issued_item - 1) & 1); ++i) {}
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(kTile, kTile);
-      bool ok = mbar_wait(smem_u32(&aux->fixed_full), 0, abort_flag);
-      for (int it = 0; ok && it < n_iter; ++it) {
-        const int st = it % kStages, b = it % kBufs;
-        ok = mbar_wait(smem_u32(&aux->full[st]), (it / kStages) & 1, abort_flag) &&
-             mbar_wait(smem_u32(&aux->acc_empty[b]), ((it / kBufs) & 1) ^ 1, abort_flag);
+      int n_item = 0, n_stream = 0, cnt[2] = {0, 0};
+      bool ok = true;
+      while (ok) {
+        const int slot = n_item & 1;
+        ok = mbar_wait(smem_u32(&aux->item_full[slot]), (n_item >> 1) & 1, abort_flag);
         if (!ok) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + b * kTile;
+        int it[5];
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = (k >> 2) * SL::kBlockBytes + (k & 3) * 32;
-          umma_bf16(d_tmem, smem_desc_sw128(fixed_addr + off), smem_desc_sw128(ring_addr + st * SL::kTileBytes + off),
-                    idesc, k > 0);
+        for (int i = 0; i < 5; ++i) it[i] = aux->item[slot][i];
+        mbar_arrive(smem_u32(&aux->item_empty[slot]));
+        if (it[0] < 0) break;
+        const Geo<kColsum> g(s, it);
+        ok = mbar_wait(smem_u32(&aux->fixed_full), n_item & 1, abort_flag);
+        for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
+          const int rs = n_stream % kRing;
+          ok = mbar_wait(smem_u32(&aux->full[rs]), (n_stream / kRing) & 1, abort_flag);
+          for (int hf = 0; ok && hf < 2; ++hf) {
+            if (!g.active(hf, i)) continue;
+            const int c = cnt[hf]++;
+            const int buf = 2 * hf + (c & 1);
+            ok = mbar_wait(smem_u32(&aux->acc_empty[buf]), ((c >> 1) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * kTile;
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+              const uint32_t off = (k >> 2) * SL::kBlockBytes + (k & 3) * 32;
+              umma_bf16(d_tmem, smem_desc_sw128(fixed_addr + hf * SL::kTileBytes + off),
+                        smem_desc_sw128(ring_addr + rs * SL::kTileBytes + off), idesc, k > 0);
+            }
+            umma_commit(smem_u32(&aux->acc_full[buf]));
+          }
+          if (!ok) break;
+          umma_commit(smem_u32(&aux->empty[rs]));
         }
-        umma_commit(smem_u32(&aux->empty[st]));
-        umma_commit(smem_u32(&aux->acc_full[b]));
+        if (!ok) break;
+        umma_commit(smem_u32(&aux->fixed_empty));
+        ++n_item;
       }
-      if (!ok) {
+      if (*abort_flag) {
         // wait (bounded) until every MMA already issued has retired before TMEM and shared memory go away
         umma_commit(smem_u32(&aux->drain));
         for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->drain), 0); ++i) {}
@@ -207,106 +282,132 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
   } else {
     // ------------------------------ epilogue groups ------------------------------
-    const int g = (warp - 2) >> 2;                 // epilogue group of this warp
+    const int gi = (warp - 2) >> 2;                // group = half * 2 + parity
+    const int hf = gi >> 1, par = gi & 1;
     const int quarter = warp & 3;                  // TMEM lanes this warp may read
-    const int r = quarter * 32 + lane;             // row of the accumulator tile = TMEM lane
-    const int gtid = r;                            // index inside the group (0..127)
-    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const int r = quarter * 32 + lane;             // row of the accumulator = TMEM lane = index inside the group
+    const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + gi * kTile;
+    const uint32_t acc_full = smem_u32(&aux->acc_full[gi]), acc_empty = smem_u32(&aux->acc_empty[gi]);
     const float scale = a.scale_log2;
     const f32x2 scale2 = splat2(scale);
+    const float ninf = __int_as_float(0xFF800000);
+    int n_item = 0, cnt = 0, n_gsync = 0, n_psync = 0;
     bool ok = true;
 
-    if constexpr (kColsum) {
-      const float* lse_row = a.lse + ((size_t)layer * s.Hq + h) * s.T + t0;
-      const float ninf = __int_as_float(0xFF800000);
-      auto load_lse = [&](int it) {                 // minus lse2 of this thread's query of streamed tile `it` (-inf past the end)
-        const int j = (first_stream + it) * kTile + gtid;
-        return (it < n_iter && j < L) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
-      };
-      f32x2 acc[2] = {0ull, 0ull};
-      float lse_next = load_lse(g);
-      int n_mine = 0;
-      for (int it = g; it < n_iter; it += kGroups, ++n_mine) {
-        const int b = it % kBufs;                   // TMEM accumulator of this tile
-        float* lse_buf = aux->lse_sh[g][n_mine & 1];
-        lse_buf[gtid] = lse_next;
-        lse_next = load_lse(it + kGroups);          // in flight while this tile is processed
-        named_bar_sync(1 + g, kEpiThreads);
-        // after a failed wait the loop keeps running (every thread must reach every named barrier) but
-        // touches neither barriers nor TMEM; `ok` is made warp-uniform because tcgen05.ld is warp-wide
-        if (ok) ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it / kBufs) & 1, abort_flag);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) continue;
-        tc_fence_after();
-        auto release = [&]() {                      // accumulator drained: hand it back to the MMA warp
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&aux->acc_empty[b]));
+    // barrier among the 4 warps of the group / the 8 warps of the half; bounded like every other wait
+    auto group_sync = [&]() {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&aux->group_bar[gi]));
+      ok = mbar_wait(smem_u32(&aux->group_bar[gi]), n_gsync & 1, abort_flag) && ok;
+      ++n_gsync;
+    };
+    auto pair_sync = [&]() {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&aux->pair_bar[hf]));
+      ok = mbar_wait(smem_u32(&aux->pair_bar[hf]), n_psync & 1, abort_flag) && ok;
+      ++n_psync;
+    };
+    auto release = [&]() {                         // accumulator drained: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty);
+    };
+
+    while (true) {
+      const int slot = n_item & 1;
+      ok = mbar_wait(smem_u32(&aux->item_full[slot]), (n_item >> 1) & 1, abort_flag) && ok;
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      int it[5];
+#pragma unroll
+      for (int i = 0; i < 5; ++i) it[i] = aux->item[slot][i];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&aux->item_empty[slot]));
+      if (it[0] < 0) break;
+      const Geo<kColsum> g(s, it);
+      const int row = g.blk * kBlockRows + hf * kTile + r;          // token of this thread inside the sequence
+      const size_t out = ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0 + row;
+
+      if constexpr (kColsum) {
+        const float* lse_row = a.lse + ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0;
+        auto load_lse = [&](int i) {                // minus lse2 of this thread's query of streamed tile i (-inf past the end)
+          const int j = (g.first_stream + i) * kTile + r;
+          return (i < g.n_iter && j < g.L) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
         };
-        const uint32_t t_acc = t_lane + b * kTile;
-        if (s.causal && it == 0)
-          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
-        else
-          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
-      }
-      float total = sum4(acc);
-      if constexpr (kGroups > 1) {
-        if (g > 0) aux->part[g][0][r] = total;
-        named_bar_sync(1 + kGroups, kGroups * kEpiThreads);
-        if (g == 0)
-          for (int o = 1; o < kGroups; ++o) total += aux->part[o][0][r];
-      }
-      if (g == 0 && ok && !*abort_flag) {
-        const int t = my_tile * kTile + r;
-        if (t < L) {
-          if (a.normalize) total = total / (float)L;
-          a.scores[((size_t)layer * s.Hq + h) * s.T + t0 + t] = total;
+        f32x2 acc[2] = {0ull, 0ull};
+        // this group's tiles of the item: every other active tile, starting where the running parity says
+        int first = g.causal ? hf : 0;
+        if (((cnt & 1) != par)) ++first;
+        float lse_next = load_lse(first);
+        int n_mine = 0;
+        for (int i = 0; i < g.n_iter && ok; ++i) {
+          if (!g.active(hf, i)) continue;
+          const int c = cnt++;
+          if ((c & 1) != par) continue;
+          float* lse_buf = aux->lse_sh[gi][n_mine & 1];
+          ++n_mine;
+          lse_buf[r] = lse_next;
+          lse_next = load_lse(i + 2);               // in flight while this tile is processed
+          group_sync();
+          ok = mbar_wait(acc_full, (c >> 1) & 1, abort_flag) && ok;
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          if (g.diag(hf, i))
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
+          else
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
         }
-      }
-    } else {
-      float m = __int_as_float(0xFF800000);                   // running max (log2 domain) of this row
-      f32x2 sum2[2] = {0ull, 0ull};                           // packed partial sums of 2^(x - m)
-      for (int it = g; it < n_iter; it += kGroups) {
-        const int b = it % kBufs;
-        ok = mbar_wait(smem_u32(&aux->acc_full[b]), (it / kBufs) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
-        tc_fence_after();
-        auto release = [&]() {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&aux->acc_empty[b]));
-        };
-        const uint32_t t_acc = t_lane + b * kTile;
-        // keys of this tile that count for this row: up to the diagonal (causal) and inside the sequence
-        const int n_valid = s.causal ? (it == my_tile ? r + 1 : kTile) : min(kTile, L - it * kTile);
-        if (__any_sync(0xFFFFFFFFu, n_valid < kTile))
-          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, scale2, n_valid - p * 16, m, sum2); }, release);
-        else
-          sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, scale2, 16, m, sum2); }, release);
-      }
-      float sum = sum4(sum2);
-      if constexpr (kGroups > 1) {
-        if (g > 0) { aux->part[g][0][r] = m; aux->part[g][1][r] = sum; }
-        named_bar_sync(1 + kGroups, kGroups * kEpiThreads);
-        if (g == 0) {                               // merge the other groups' (max, sum)
-          for (int o = 1; o < kGroups; ++o) {
-            const float m1 = aux->part[o][0][r], sum1 = aux->part[o][1][r];
-            const float big = fmaxf(m, m1);
-            sum = sum * ex2(m - big) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
-            m = big;
-          }
+        float total = sum4(acc);
+        float* part = aux->part[hf][n_item & 1][0];
+        if (par == 1) part[r] = total;
+        pair_sync();
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        if (par == 0 && row < g.L && (hf == 0 || g.half1)) {
+          total += part[r];
+          if (a.normalize) total = total / (float)g.L;
+          a.scores[out] = total;
+        }
+      } else {
+        float m = __int_as_float(0xFF800000);                   // running max (log2 domain) of this row
+        f32x2 sum2[2] = {0ull, 0ull};                           // packed partial sums of 2^(x - m)
+        for (int i = 0; i < g.n_iter && ok; ++i) {
+          if (!g.active(hf, i)) continue;
+          const int c = cnt++;
+          if ((c & 1) != par) continue;
+          ok = mbar_wait(acc_full, (c >> 1) & 1, abort_flag) && ok;
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          // keys of this tile that count for this row: up to the diagonal (causal) and inside the sequence
+          const int n_valid = g.causal ? (g.diag(hf, i) ? r + 1 : kTile) : min(kTile, g.L - i * kTile);
+          if (__any_sync(0xFFFFFFFFu, n_valid < kTile))
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, scale2, n_valid - p * 16, m, sum2); }, release);
+          else
+            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, scale2, 16, m, sum2); }, release);
+        }
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        const float sum = sum4(sum2);
+        float* pm = aux->part[hf][n_item & 1][0];
+        float* ps = aux->part[hf][n_item & 1][1];
+        if (par == 1) { pm[r] = m; ps[r] = sum; }
+        pair_sync();
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        if (par == 0 && row < g.L && (hf == 0 || g.half1)) {       // merge the other group's (max, sum)
+          const float m1 = pm[r], sum1 = ps[r];
+          const float big = fmaxf(m, m1);
+          const float tot = (sum > 0.f ? sum * ex2(m - big) : 0.f) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
+          const float lse2 = big + log2f(tot);
+          a.lse2_out[out] = lse2;
+          if (a.lse_nat_out) a.lse_nat_out[out] = lse2 * 0.69314718055994530942f;
         }
       }
-      if (g == 0 && ok && !*abort_flag) {
-        const int j = my_tile * kTile + r;
-        if (j < L) {
-          const float lse2 = m + log2f(sum);
-          const size_t o = ((size_t)layer * s.Hq + h) * s.T + t0 + j;
-          a.lse2_out[o] = lse2;
-          if (a.lse_nat_out) a.lse_nat_out[o] = lse2 * 0.69314718055994530942f;
-        }
-      }
+      ++n_item;
     }
   }
 
@@ -319,25 +420,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   if (tid == 0 && !dead && *abort_flag) report(a.status, KVCRUSH_DEV_TIMEOUT, kColsum ? KID_SCORE_COLSUM : KID_SCORE_LSE, blockIdx.x, 0);
 }
 
-// ------------------------------------------------------------------------------------------------
-// host side
-// ------------------------------------------------------------------------------------------------
 template <int D, bool kColsum>
-int launch_sweep(const CUtensorMap& mq, const CUtensorMap& mk, const ScoreArgs& a, cudaStream_t stream) {
-  auto kern = score_tc_kernel<D, kColsum>;
-  constexpr int smem = SmemLayout<D>::kTotal;
-  static bool configured = false;      // per process; the attribute is idempotent, so a race only repeats the call
-  if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return KVCRUSH_ERR_CUDA;
-    configured = true;
-  }
-  const long long blocks = (long long)a.n_items * a.s.n_layers * a.s.Hq;
-  if (blocks > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
+int launch_persist(const CUtensorMap& mq, const CUtensorMap& mk, const PersistArgs& a, int n_sms, cudaStream_t stream) {
+  auto kern = score_persist_kernel<D, kColsum>;
+  constexpr int smem = PSmem<D>::kTotal;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return KVCRUSH_ERR_CUDA;
+  const int blocks = a.total_items < n_sms ? a.total_items : n_sms;
   kern<<<(unsigned)blocks, kThreads, smem, stream>>>(mq, mk, a);
   return check_launch();
 }
 
 }  // namespace
+
+size_t score_tensor_counter_bytes() { return 256; }
 
 bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorView& K) {
   if (Q.dtype != KVCRUSH_BF16 || K.dtype != KVCRUSH_BF16) return false;
@@ -346,32 +441,42 @@ bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorVie
   return encode_fn() != nullptr;
 }
 
+
 int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView& Q, const TensorView& K,
-                        float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores,
-                        float* lse_out, int normalize, int32_t* status, cudaStream_t stream) {
-  static_assert(sizeof(Aux) <= 12288, "aux block too large");
+                                   float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws,
+                                   int* counters, float* scores, float* lse_out, int normalize, int32_t* status,
+                                   cudaStream_t stream) {
+  static_assert(sizeof(PAux) <= 10240, "aux block too large");
   if (!(scale_log2 > 0.f)) return KVCRUSH_ERR_UNSUPPORTED;
   CUtensorMap mq, mk;
   if (!make_map(&mq, Q, s.D, s.T, s.Hq, s.n_layers) || !make_map(&mk, K, s.D, s.T, s.Hkv, s.n_layers))
     return KVCRUSH_ERR_CUDA;
-  ScoreArgs a{};
+  int dev = 0, n_sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sms < 1)
+    return KVCRUSH_ERR_CUDA;
+  PersistArgs a{};
   a.s = s; a.scale_log2 = scale_log2; a.normalize = normalize; a.status = status; a.scores = scores;
-  a.max_tiles = (s.max_seqlen + kTile - 1) / kTile;
+  a.max_blocks = (s.max_seqlen + kBlockRows - 1) / kBlockRows;
   long long items = 0;
-  for (int i = 0; i < s.n_seqs; ++i) items += (cu_host[i + 1] - cu_host[i] + kTile - 1) / kTile;
+  for (int i = 0; i < s.n_seqs; ++i) items += (cu_host[i + 1] - cu_host[i] + kBlockRows - 1) / kBlockRows;
   if (items == 0) return KVCRUSH_OK;
-  if (items > 0x7FFFFFFF) return KVCRUSH_ERR_UNSUPPORTED;
+  const long long total = items * s.n_layers * s.Hq;
+  if (total > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
   a.n_items = (int)items;
+  a.total_items = (int)total;
+  if (cudaMemsetAsync(counters, 0, 2 * sizeof(int), stream) != cudaSuccess) return KVCRUSH_ERR_CUDA;
   int rc;
   if (!lse_in) {
-    a.lse2_out = lse2_ws; a.lse_nat_out = lse_out;
-    rc = s.D == 128 ? launch_sweep<128, false>(mq, mk, a, stream) : launch_sweep<64, false>(mq, mk, a, stream);
+    a.lse2_out = lse2_ws; a.lse_nat_out = lse_out; a.counter = counters;
+    rc = s.D == 128 ? launch_persist<128, false>(mq, mk, a, n_sms, stream) : launch_persist<64, false>(mq, mk, a, n_sms, stream);
     if (rc != KVCRUSH_OK) return rc;
     a.lse = lse2_ws; a.lse_mul = 1.f;
   } else {
     a.lse = lse_in; a.lse_mul = lse_in_mul;
   }
-  return s.D == 128 ? launch_sweep<128, true>(mq, mk, a, stream) : launch_sweep<64, true>(mq, mk, a, stream);
+  a.counter = counters + 1;
+  return s.D == 128 ? launch_persist<128, true>(mq, mk, a, n_sms, stream) : launch_persist<64, true>(mq, mk, a, n_sms, stream);
 }
 
 }  // namespace kvc

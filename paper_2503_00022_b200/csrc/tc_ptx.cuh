@@ -79,9 +79,6 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void named_bar_sync(int id, int n) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
-}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -145,15 +142,19 @@ __device__ __forceinline__ f32x2 exp2_poly2(f32x2 x) {
   return pack2(__float_as_uint(p0) + (__float_as_uint(t0) << 23), __float_as_uint(p1) + (__float_as_uint(t1) << 23));
 }
 
-#ifndef KVC_POLY_PAIRS_PER4
-#define KVC_POLY_PAIRS_PER4 1                        // of every 4 pairs of exponentials, this many use exp2_poly2
+// Share of the exponentials that takes the FMA-pipe path, in pairs out of every 4 pairs, per sweep.
+// Measured under the board power limit (32 layers x 32 heads x 8192 tokens): the row sweep is fastest
+// with none, the column sweep with one pair in four.
+#ifndef KVC_POLY_PAIRS_LSE
+#define KVC_POLY_PAIRS_LSE 0
 #endif
-__host__ __device__ constexpr bool poly_pair(int j) {
-  return ((j % 4 + 1) * KVC_POLY_PAIRS_PER4) / 4 > ((j % 4) * KVC_POLY_PAIRS_PER4) / 4;
-}
-template <int J>
+#ifndef KVC_POLY_PAIRS_COLSUM
+#define KVC_POLY_PAIRS_COLSUM 1
+#endif
+template <int J, int P>
 __device__ __forceinline__ f32x2 exp2_mix2(f32x2 x) {
-  if constexpr (poly_pair(J)) return exp2_poly2(x); else return exp2_sfu2(x);
+  constexpr bool poly = ((J % 4 + 1) * P) / 4 > ((J % 4) * P) / 4;
+  if constexpr (poly) return exp2_poly2(x); else return exp2_sfu2(x);
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -204,7 +205,7 @@ __device__ __forceinline__ void sweep_tile(uint32_t taddr, Piece&& piece, Releas
 // nlse16: MINUS the log2-domain row log-sum-exp of the 16 queries (-inf past the end of the sequence).
 template <int J, bool kDiag>
 __device__ __forceinline__ f32x2 colsum_pair(uint32_t v0, uint32_t v1, float nl0, float nl1, f32x2 scale2, int r, int c) {
-  f32x2 e = exp2_mix2<J>(fma2(pack2(v0, v1), scale2, pack2f(nl0, nl1)));
+  f32x2 e = exp2_mix2<J, KVC_POLY_PAIRS_COLSUM>(fma2(pack2(v0, v1), scale2, pack2f(nl0, nl1)));
   if constexpr (kDiag) {                            // causal: the query (column) must not precede the key (row)
     float e0, e1;
     unpack2(e, e0, e1);
@@ -254,14 +255,14 @@ __device__ __forceinline__ void lse_piece(const uint32_t (&v)[16], float scale, 
     m = m_new;
   }
   const f32x2 nm = splat2(-m);
-  sum2[0] = add2(sum2[0], exp2_mix2<0>(fma2(pack2(x[0], x[1]), scale2, nm)));
-  sum2[1] = add2(sum2[1], exp2_mix2<1>(fma2(pack2(x[2], x[3]), scale2, nm)));
-  sum2[0] = add2(sum2[0], exp2_mix2<2>(fma2(pack2(x[4], x[5]), scale2, nm)));
-  sum2[1] = add2(sum2[1], exp2_mix2<3>(fma2(pack2(x[6], x[7]), scale2, nm)));
-  sum2[0] = add2(sum2[0], exp2_mix2<0>(fma2(pack2(x[8], x[9]), scale2, nm)));
-  sum2[1] = add2(sum2[1], exp2_mix2<1>(fma2(pack2(x[10], x[11]), scale2, nm)));
-  sum2[0] = add2(sum2[0], exp2_mix2<2>(fma2(pack2(x[12], x[13]), scale2, nm)));
-  sum2[1] = add2(sum2[1], exp2_mix2<3>(fma2(pack2(x[14], x[15]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<0, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[0], x[1]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<1, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[2], x[3]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<2, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[4], x[5]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<3, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[6], x[7]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<0, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[8], x[9]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<1, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[10], x[11]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<2, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[12], x[13]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<3, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[14], x[15]), scale2, nm)));
 }
 __device__ __forceinline__ float sum4(const f32x2 (&s)[2]) {
   float a, b, c, d;
