@@ -210,6 +210,10 @@ TENSOR_CASES = [
     inputs.Workload("tc_d64", 1, 4, 2, 64, (513, 64), inputs.BF16, inputs.BF16, 0.25, base_seed=34),
     inputs.Workload("tc_noncausal", 1, 4, 4, 128, (333, 260), inputs.BF16, inputs.BF16, 0.25, base_seed=35, causal=False),
     inputs.Workload("tc_2k", 1, 8, 8, 128, (2048,), inputs.BF16, inputs.BF16, 0.25, base_seed=36),
+    # more sequences than one warp decodes at once, lengths around every tile / block boundary, an empty sequence
+    inputs.Workload("tc_many_seqs", 1, 2, 1, 64, tuple([127, 128, 129, 255, 256, 257, 0, 1, 383, 384, 385, 512] * 3 + [40, 300]),
+                    inputs.BF16, inputs.BF16, 0.25, base_seed=37),
+    inputs.Workload("tc_128_heads", 1, 128, 16, 64, (260,), inputs.BF16, inputs.BF16, 0.25, base_seed=38),
 ]
 
 
@@ -246,3 +250,31 @@ def test_score_tensor_rejects_fp32_and_auto_falls_back_to_cuda_cores(B):
     B.kvcrush_score(prob, dq, dk, scores, impl=B.SCORE_AUTO, workspace=ws, status=status)
     torch.cuda.synchronize()
     assert torch.isfinite(scores).all()
+
+
+@pytest.mark.parametrize("impl_name", ["SCORE_TENSOR", "SCORE_SIMT"])
+def test_score_head_major_layout_and_explicit_scale(B, impl_name):
+    """Q/K stored [layer, head, token, D] (reached through strides) and a caller-chosen softmax scale."""
+    import torch
+    dev = _dev()
+    impl = getattr(B, impl_name)
+    w = inputs.Workload("hm", 2, 4, 2, 128, (391, 130), inputs.BF16, inputs.BF16, 0.25, base_seed=41)
+    lis, q, k, _, _ = TL.stack_layers(w, range(2), with_cache=False)
+    scale = 0.05
+    prob = B.Problem(2, 4, 2, 128, w.seqlens, causal=True, softmax_scale=scale, device=dev)
+    dq = TL.torch_storage(q, w.qk_dtype, dev).permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    dk = TL.torch_storage(k, w.qk_dtype, dev).permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert dq.stride(1) == 128 and dq.stride(2) == 128 * w.total_tokens
+    scores = torch.empty((2, 4, w.total_tokens), dtype=torch.float32, device=dev)
+    ws = torch.empty(B.kvcrush_workspace_size(prob, B.STAGE_SCORE), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    B.kvcrush_score(prob, dq, dk, scores, impl=impl, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0
+    g = scores.cpu().numpy()
+    cu = w.cu_seqlens
+    for l, li in enumerate(lis):
+        for s_, L in enumerate(w.seqlens):
+            a, b = int(cu[s_]), int(cu[s_ + 1])
+            c, _ = O.scores(inputs.widen(li.q[a:b], w.qk_dtype), inputs.widen(li.k[a:b], w.qk_dtype), True, scale=scale)
+            assert TL.within_score_tolerance(g[l][:, a:b], c).all()
