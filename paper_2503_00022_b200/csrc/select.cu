@@ -57,6 +57,8 @@ struct SelectArgs {
   uint8_t* kind;
   int32_t* sorted;                    // [n_layers][T] scratch: grouped tokens in (d, t) order
   int mask_words;                     // words of one membership mask in shared memory
+  int stage_words;                    // max_seqlen rounded up to a multiple of 4 (one staged int32 per token)
+  int stage_sorted, stage_sig, stage_keys;   // which per-segment arrays are copied into shared memory
 };
 
 __device__ __forceinline__ uint32_t head_mask(int Hq, int w) {
@@ -64,7 +66,8 @@ __device__ __forceinline__ uint32_t head_mask(int Hq, int w) {
   return n >= 32 ? 0xFFFFFFFFu : ((1u << n) - 1u);
 }
 
-__global__ void __launch_bounds__(kThreads)
+template <int W>                       // signature words per token (compile time: the per-word loops unroll)
+__global__ void __launch_bounds__(kThreads, 1)
 select_segment_kernel(Shape s, SelectArgs a) {
   extern __shared__ uint32_t dyn_smem[];
   uint32_t* imp_mask = dyn_smem;
@@ -98,9 +101,26 @@ select_segment_kernel(Shape s, SelectArgs a) {
     return;
   }
 
+  // The segment's arrays are read many times with dependent addresses (8 radix sweeps, two counting-sort
+  // sweeps, one gather per bucket), so whatever fits is first copied into shared memory; the rest is read
+  // through L2.  The pointers below are generic and point to either place.
   const unsigned long long* keys = a.keys + (size_t)layer * s.T + t0;
-  const uint32_t* sig = a.sigs + ((size_t)layer * s.T + t0) * s.W;
+  const uint32_t* sig = a.sigs + ((size_t)layer * s.T + t0) * W;
   int32_t* sorted = a.sorted + (size_t)layer * s.T + t0;
+  {
+    uint32_t* arena = dyn_smem + 2 * a.mask_words;
+    if (a.stage_sorted) { sorted = reinterpret_cast<int32_t*>(arena); arena += a.stage_words; }
+    if (a.stage_sig) {
+      for (int i = tid; i < L * W; i += kThreads) arena[i] = __ldg(sig + i);
+      sig = arena;
+      arena += a.stage_words * W;
+    }
+    if (a.stage_keys) {
+      unsigned long long* ks = reinterpret_cast<unsigned long long*>(arena);
+      for (int i = tid; i < L; i += kThreads) ks[i] = keys[i];
+      keys = ks;
+    }
+  }
   const int n_words = (L + 31) >> 5;
   // contiguous token range of this warp (multiple of 32 tokens so that mask words do not straddle)
   const int per_warp = ((n_words + kWarps - 1) / kWarps) * 32;
@@ -120,13 +140,19 @@ select_segment_kernel(Shape s, SelectArgs a) {
       for (int base = 0; base < L; base += kThreads) {
         const int i = base + tid;
         const bool in = i < L;
-        const unsigned long long key = in ? __ldg(keys + i) : 0ull;
+        const unsigned long long key = in ? keys[i] : 0ull;
         const bool live = in && ((key & hi_mask) == prefix);
         const uint32_t digit = (uint32_t)(key >> shift) & 0xFFu;
+        // high digits (sign, exponent) are the same for almost every key: one add per warp then;
+        // low digits are spread over the 256 bins, where plain shared-memory atomics do not collide much
         const unsigned voters = __ballot_sync(kFull, live);
-        if (live) {
-          const unsigned peers = __match_any_sync(voters, digit);
-          if ((peers & lt_mask) == 0) atomicAdd(&hist[digit], __popc(peers));
+        if (voters) {
+          const uint32_t d0 = __shfl_sync(kFull, digit, __ffs(voters) - 1);
+          if (__all_sync(kFull, !live || digit == d0)) {
+            if (lane == 0) atomicAdd(&hist[d0], __popc(voters));
+          } else if (live) {
+            atomicAdd(&hist[digit], 1u);
+          }
         }
       }
       __syncthreads();
@@ -162,7 +188,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
     // prefix = the b_imp-th largest key; k_rem = how many keys equal to it are admitted
     const unsigned long long kth = prefix;
     int n_eq = 0;
-    for (int i = r_lo + lane; i < r_hi; i += 32) n_eq += (__ldg(keys + i) == kth);
+    for (int i = r_lo + lane; i < r_hi; i += 32) n_eq += (keys[i] == kth);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) n_eq += __shfl_xor_sync(kFull, n_eq, d);
     if (lane == 0) warp_tot[warp] = n_eq;
@@ -171,7 +197,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
     for (int w = 0; w < warp; ++w) eq_before += warp_tot[w];
     for (int base = r_lo; base < r_hi; base += 32) {
       const int i = base + lane;
-      const unsigned long long key = i < r_hi ? __ldg(keys + i) : 0ull;
+      const unsigned long long key = i < r_hi ? keys[i] : 0ull;
       const bool eq = i < r_hi && key == kth;
       const unsigned eq_b = __ballot_sync(kFull, eq);
       const bool imp = i < r_hi && (key > kth || (eq && (uint32_t)(eq_before + __popc(eq_b & lt_mask)) < k_rem));
@@ -185,7 +211,6 @@ select_segment_kernel(Shape s, SelectArgs a) {
   // ---- 2-4. representatives of the other tokens ------------------------------------------------
   if (b_rep > 0) {
     const int N = L - b_imp;
-    const int W = s.W;
     // anchor
     if (a.anchor_mode == KVCRUSH_ANCHOR_MEAN) {
       for (int i = tid; i < 128; i += kThreads) bit_cnt[i] = 0;
@@ -194,8 +219,8 @@ select_segment_kernel(Shape s, SelectArgs a) {
       for (int base = r_lo; base < r_hi; base += 32) {
         const int i = base + lane;
         const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
-        for (int w = 0; w < W; ++w) {
-          const uint32_t word = cand ? __ldg(sig + (size_t)i * W + w) : 0u;
+        _Pragma("unroll") for (int w = 0; w < W; ++w) {
+          const uint32_t word = cand ? sig[(size_t)i * W + w] : 0u;
           const int nb = min(32, s.Hq - 32 * w);
           for (int b = 0; b < nb; ++b) {
             const unsigned m = __ballot_sync(kFull, (word >> b) & 1u);
@@ -203,7 +228,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
           }
         }
       }
-      for (int w = 0; w < W; ++w)
+      _Pragma("unroll") for (int w = 0; w < W; ++w)
         if (32 * w + lane < s.Hq && acc[w]) atomicAdd(&bit_cnt[32 * w + lane], acc[w]);
       __syncthreads();
       if (warp < W) {
@@ -222,7 +247,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
     for (int i = tid; i < kWarps * kMaxBins; i += kThreads) (&warp_hist[0][0])[i] = 0;
     __syncthreads();
     uint32_t anc[4], hm[4];
-    for (int w = 0; w < 4; ++w) { anc[w] = w < W ? anchor_sh[w] : 0u; hm[w] = w < W ? head_mask(s.Hq, w) : 0u; }
+    _Pragma("unroll") for (int w = 0; w < 4; ++w) { anc[w] = w < W ? anchor_sh[w] : 0u; hm[w] = w < W ? head_mask(s.Hq, w) : 0u; }
     const int n_bins = s.Hq + 1;
 
     // counting sort by (d, t): per-warp histograms over contiguous token ranges
@@ -231,7 +256,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
       const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
       int d = 0;
       if (cand)
-        for (int w = 0; w < W; ++w) d += __popc((__ldg(sig + (size_t)i * W + w) ^ anc[w]) & hm[w]);
+        _Pragma("unroll") for (int w = 0; w < W; ++w) d += __popc((sig[(size_t)i * W + w] ^ anc[w]) & hm[w]);
       const unsigned voters = __ballot_sync(kFull, cand);
       if (cand) {
         const unsigned peers = __match_any_sync(voters, d);
@@ -256,7 +281,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
       const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
       int d = 0;
       if (cand)
-        for (int w = 0; w < W; ++w) d += __popc((__ldg(sig + (size_t)i * W + w) ^ anc[w]) & hm[w]);
+        _Pragma("unroll") for (int w = 0; w < W; ++w) d += __popc((sig[(size_t)i * W + w] ^ anc[w]) & hm[w]);
       const unsigned voters = __ballot_sync(kFull, cand);
       unsigned peers = 0;
       if (cand) {
@@ -270,31 +295,43 @@ select_segment_kernel(Shape s, SelectArgs a) {
     __syncthreads();
 
     // one representative per equal-frequency bucket (one warp per bucket)
+    // bucket i covers sorted positions [floor(i*N/R), floor((i+1)*N/R)).  64-bit divisions are slow, so each
+    // warp divides once and then steps exactly: i*N = pos*R + rem, and the stride kWarps*N = step_q*R + step_r.
+    const int q_nr = N / b_rep, r_nr = N - q_nr * b_rep;                       // N = q_nr*R + r_nr
+    const long long stride = (long long)kWarps * N;
+    const int step_q = (int)(stride / b_rep), step_r = (int)(stride - (long long)step_q * b_rep);
+    int pos = (int)(((long long)warp * N) / b_rep);
+    int rem = (int)((long long)warp * N - (long long)pos * b_rep);
     for (int bkt = warp; bkt < b_rep; bkt += kWarps) {
-      const int lo = (int)(((long long)bkt * N) / b_rep);
-      const int hi = (int)(((long long)(bkt + 1) * N) / b_rep);
+      const int lo = pos;
+      const int hi = pos + q_nr + (rem + r_nr >= b_rep ? 1 : 0);
       const int m = hi - lo;
+      pos += step_q;
+      rem += step_r;
+      if (rem >= b_rep) { rem -= b_rep; ++pos; }
       unsigned long long best = ~0ull;
       if (m <= 32) {
+        // one lane per member.  sum_{h set in t} n_h = sum over members u of popc(sig_t & sig_u), so
+        // cost(t) = m * popc(sig_t) - 2 * sum_u popc(sig_t & sig_u): m shuffles instead of one ballot per head
         const bool member = lane < m;
         const int t = member ? sorted[lo + lane] : 0;
-        int cost = 0;
-        for (int w = 0; w < W; ++w) {
-          const uint32_t word = member ? __ldg(sig + (size_t)t * W + w) : 0u;
-          const int nb = min(32, s.Hq - 32 * w);
-          for (int b = 0; b < nb; ++b) {
-            const unsigned ones = __ballot_sync(kFull, (word >> b) & 1u);
-            if ((word >> b) & 1u) cost += m - 2 * __popc(ones);
-          }
+        uint32_t mine[4] = {0u, 0u, 0u, 0u};
+        _Pragma("unroll") for (int w = 0; w < W; ++w) mine[w] = member ? sig[(size_t)t * W + w] & head_mask(s.Hq, w) : 0u;
+        int ones = 0, shared = 0;
+        _Pragma("unroll") for (int w = 0; w < W; ++w) ones += __popc(mine[w]);
+        for (int u0 = 0; u0 < m; u0 += 4) {        // lanes >= m hold zeros, so reading past m adds nothing
+          _Pragma("unroll") for (int du = 0; du < 4; ++du)
+            _Pragma("unroll") for (int w = 0; w < W; ++w) shared += __popc(mine[w] & __shfl_sync(kFull, mine[w], (u0 + du) & 31));
         }
+        const int cost = m * ones - 2 * shared;
         if (member) best = ((unsigned long long)((uint32_t)cost + 0x80000000u) << 32) | (uint32_t)t;
       } else {
         int n_ones[4] = {0, 0, 0, 0};        // lane b of word w holds n_h for head 32w+b
         for (int c0 = lo; c0 < hi; c0 += 32) {
           const bool member = c0 + lane < hi;
           const int t = member ? sorted[c0 + lane] : 0;
-          for (int w = 0; w < W; ++w) {
-            const uint32_t word = member ? __ldg(sig + (size_t)t * W + w) : 0u;
+          _Pragma("unroll") for (int w = 0; w < W; ++w) {
+            const uint32_t word = member ? sig[(size_t)t * W + w] : 0u;
             const int nb = min(32, s.Hq - 32 * w);
             for (int b = 0; b < nb; ++b) {
               const unsigned ones = __ballot_sync(kFull, (word >> b) & 1u);
@@ -306,8 +343,8 @@ select_segment_kernel(Shape s, SelectArgs a) {
           const bool member = c0 + lane < hi;
           const int t = member ? sorted[c0 + lane] : 0;
           int cost = 0;
-          for (int w = 0; w < W; ++w) {
-            const uint32_t word = member ? __ldg(sig + (size_t)t * W + w) : 0u;
+          _Pragma("unroll") for (int w = 0; w < W; ++w) {
+            const uint32_t word = member ? sig[(size_t)t * W + w] : 0u;
             const int nb = min(32, s.Hq - 32 * w);
             for (int b = 0; b < nb; ++b) {
               const int n_h = __shfl_sync(kFull, n_ones[w], b);
@@ -384,13 +421,30 @@ int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, con
   a.anchor_mode = anchor_mode; a.anchor_bits = anchor_bits; a.anchor_per_segment = anchor_per_segment;
   a.cu_kept = cu_kept; a.idx = idx; a.kind = kind; a.sorted = sorted;
   a.mask_words = ((s.max_seqlen + 31) / 32 + 3) & ~3;
-  const size_t dyn = (size_t)a.mask_words * 2 * sizeof(uint32_t);
+  a.stage_words = (s.max_seqlen + 3) & ~3;
+  size_t dyn = (size_t)a.mask_words * 2 * sizeof(uint32_t);
+  const size_t budget = 196 * 1024;     // dynamic shared memory this kernel may take (static part: ~19 KB)
+  const size_t per_tok = (size_t)a.stage_words * sizeof(uint32_t);
+  if (dyn + per_tok <= budget) { a.stage_sorted = 1; dyn += per_tok; }
+  if (dyn + per_tok * s.W <= budget) { a.stage_sig = 1; dyn += per_tok * s.W; }
+  if (dyn + 2 * per_tok <= budget) { a.stage_keys = 1; dyn += 2 * per_tok; }
   if (dyn > 16 * 1024) {     // static + dynamic shared memory above the 48 KB default needs the opt-in
-    if (cudaFuncSetAttribute(select_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) !=
-        cudaSuccess)
-      return KVCRUSH_ERR_CUDA;
+    cudaError_t e = cudaSuccess;
+    switch (s.W) {
+      case 1: e = cudaFuncSetAttribute(select_segment_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); break;
+      case 2: e = cudaFuncSetAttribute(select_segment_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); break;
+      case 3: e = cudaFuncSetAttribute(select_segment_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); break;
+      default: e = cudaFuncSetAttribute(select_segment_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); break;
+    }
+    if (e != cudaSuccess) return KVCRUSH_ERR_CUDA;
   }
-  select_segment_kernel<<<(unsigned)(s.n_layers * s.n_seqs), kThreads, dyn, stream>>>(s, a);
+  const unsigned n_seg = (unsigned)(s.n_layers * s.n_seqs);
+  switch (s.W) {
+    case 1: select_segment_kernel<1><<<n_seg, kThreads, dyn, stream>>>(s, a); break;
+    case 2: select_segment_kernel<2><<<n_seg, kThreads, dyn, stream>>>(s, a); break;
+    case 3: select_segment_kernel<3><<<n_seg, kThreads, dyn, stream>>>(s, a); break;
+    default: select_segment_kernel<4><<<n_seg, kThreads, dyn, stream>>>(s, a); break;
+  }
   return check_launch();
 }
 

@@ -2,7 +2,7 @@
 //
 //   theta_select_kernel   theta = keep-th largest score of one (layer, sequence, head): an exact
 //                         MSB-first radix select over order-preserving 32-bit keys (4 sweeps of 8
-//                         bits, warp-aggregated shared-memory histograms).
+//                         bits, shared-memory histograms with a one-add-per-warp path for uniform digits).
 //   binarise_pack_kernel  one thread per (layer, token): compares the token's score of every head
 //                         with that head's threshold and packs the bits.  Lanes are consecutive
 //                         tokens, so every per-head load is a coalesced 128-byte row.
@@ -55,10 +55,16 @@ theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __
       const uint32_t key = in ? order_key(__ldg(row + i)) : 0u;
       const bool live = in && ((key & hi_mask) == prefix);
       const uint32_t digit = (key >> shift) & 0xFFu;
+      // high digits (sign, exponent) are the same for almost every score: one add per warp then;
+      // low digits are spread over the 256 bins, where plain shared-memory atomics do not collide much
       const unsigned voters = __ballot_sync(0xFFFFFFFFu, live);
-      if (live) {
-        const unsigned peers = __match_any_sync(voters, digit);
-        if ((peers & ((1u << lane) - 1u)) == 0) atomicAdd(&hist[digit], __popc(peers));
+      if (voters) {
+        const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, __ffs(voters) - 1);
+        if (__all_sync(0xFFFFFFFFu, !live || digit == d0)) {
+          if (lane == 0) atomicAdd(&hist[d0], __popc(voters));
+        } else if (live) {
+          atomicAdd(&hist[digit], 1u);
+        }
       }
     }
     __syncthreads();
