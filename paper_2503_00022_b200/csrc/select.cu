@@ -32,12 +32,21 @@ importance_kernel(Shape s, const float* __restrict__ scores, unsigned long long*
   if (gid >= (long long)s.n_layers * s.T) return;
   const int layer = (int)(gid / s.T), tok = (int)(gid - (long long)layer * s.T);
   const float* sc = scores + (size_t)layer * s.Hq * s.T + tok;
-  double total = 0.0;
-  for (int g = 0; g < s.Hkv; ++g) {
-    double group = 0.0;
-    for (int j = 0; j < s.G; ++j)
-      group = __dadd_rn(group, (double)__ldg(sc + (size_t)(g * s.G + j) * s.T));
-    total = __dadd_rn(total, group);
+  // the additions are sequential by definition (fixed order = bit-reproducible ranking); the loads are not,
+  // so they are issued eight at a time ahead of the adds that consume them
+  double total = 0.0, group = 0.0;
+  int in_group = 0;
+  for (int h0 = 0; h0 < s.Hq; h0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = h0 + j < s.Hq ? __ldg(sc + (size_t)(h0 + j) * s.T) : 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (h0 + j < s.Hq) {
+        group = __dadd_rn(group, (double)v[j]);
+        if (++in_group == s.G) { total = __dadd_rn(total, group); group = 0.0; in_group = 0; }
+      }
+    }
   }
   total = __dadd_rn(total, 0.0);           // -0.0 -> +0.0
   const unsigned long long b = (unsigned long long)__double_as_longlong(total);

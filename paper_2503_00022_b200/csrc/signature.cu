@@ -25,7 +25,8 @@ __device__ __forceinline__ float key_to_float(uint32_t k) {
 
 __global__ void __launch_bounds__(kSelectThreads)
 theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __restrict__ sig_keep,
-                    float* __restrict__ theta) {
+                    float* __restrict__ theta, int stage_row) {
+  extern __shared__ uint32_t row_keys[];          // the row's order keys when it fits (stage_row), else unused
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sel_prefix, sel_k;
 
@@ -52,7 +53,15 @@ theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __
     for (int base = 0; base < L; base += kSelectThreads) {
       const int i = base + threadIdx.x;
       const bool in = i < L;
-      const uint32_t key = in ? order_key(__ldg(row + i)) : 0u;
+      // the first sweep reads the scores and, when the row fits, leaves its keys in shared memory for the other three
+      uint32_t key = 0u;
+      if (in) {
+        if (stage_row && shift != 24) key = row_keys[i];
+        else {
+          key = order_key(__ldg(row + i));
+          if (stage_row) row_keys[i] = key;
+        }
+      }
       const bool live = in && ((key & hi_mask) == prefix);
       const uint32_t digit = (key >> shift) & 0xFFu;
       // high digits (sign, exponent) are the same for almost every score: one add per warp then;
@@ -130,7 +139,13 @@ int launch_signature(const Shape& s, const float* scores, const int32_t* sig_kee
   const float* th = theta_in;
   if (!theta_in) {
     const unsigned blocks = (unsigned)s.n_layers * s.n_seqs * s.Hq;
-    theta_select_kernel<<<blocks, kSelectThreads, 0, stream>>>(s, scores, sig_keep, theta);
+    const size_t row_bytes = (size_t)s.max_seqlen * sizeof(uint32_t);
+    const int stage_row = row_bytes <= 96 * 1024;
+    const size_t dyn = stage_row ? row_bytes : 0;
+    if (dyn > 40 * 1024 &&
+        cudaFuncSetAttribute(theta_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+      return KVCRUSH_ERR_CUDA;
+    theta_select_kernel<<<blocks, kSelectThreads, dyn, stream>>>(s, scores, sig_keep, theta, stage_row);
     if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
     th = theta;
   }
