@@ -43,6 +43,17 @@ function or parameter here):
   exactly B kept tokens;
 * the centroid is the per-bit mean and "closest" is L1 (equivalently squared
   L2) distance, evaluated as an exact integer cost (``representative``).
+
+SnapKV-style importance (Sec. 2.3 and Sec. 4.1.1 describe it in one sentence each: the
+observation window is limited to the final tokens of the prompt, and max pooling keeps
+neighbouring KVs) is covered by three small pieces, all PARITY UNPINNED by this paper
+because it gives no formula for them:
+
+* ``scores(..., rows=(L - w, L))``: only the last w queries vote;
+* ``max_pool``: every per-head score becomes the maximum over a centred window of odd
+  width (positions outside the sequence do not count);
+* ``select(..., keep_recent=n)``: the last n tokens are important by decree (their
+  importance is +inf) and count against B_important.
 """
 from __future__ import annotations
 
@@ -202,6 +213,18 @@ def importance(scores32: np.ndarray, n_kv_heads: int) -> np.ndarray:
     return total
 
 
+def max_pool(scores32: np.ndarray, kernel: int) -> np.ndarray:
+    """out[h, t] = max of scores32[h, t - r .. t + r] inside the sequence, r = (kernel - 1) / 2,
+    kernel odd (Sec. 2.3: max pooling retains the neighbours of a high-scoring token)."""
+    assert kernel >= 1 and kernel % 2 == 1
+    Hq, L = scores32.shape
+    r = (kernel - 1) // 2
+    out = np.empty_like(scores32)
+    for t in range(L):
+        out[:, t] = scores32[:, max(0, t - r):min(L, t + r + 1)].max(axis=1)
+    return out
+
+
 def top_important(I: np.ndarray, b_imp: int) -> np.ndarray:
     """Token ids of the b_imp largest I, ties to the lower index; returned ascending."""
     L = I.shape[0]
@@ -291,7 +314,8 @@ def representative(member_tokens: np.ndarray, member_sigs: np.ndarray, n_q_heads
 # ---------------------------------------------------------------------------
 
 def select(scores32: np.ndarray, sig: np.ndarray, b_imp: int, b_rep: int, n_kv_heads: int,
-           anchor_mode: int = ANCHOR_ALTERNATE, explicit_anchor: Optional[np.ndarray] = None):
+           anchor_mode: int = ANCHOR_ALTERNATE, explicit_anchor: Optional[np.ndarray] = None,
+           keep_recent: int = 0):
     """Kept token ids (ascending) and their kind (0 important, 1 representative).
 
     A budget b_imp + b_rep >= L keeps every token (kind 0)."""
@@ -299,6 +323,9 @@ def select(scores32: np.ndarray, sig: np.ndarray, b_imp: int, b_rep: int, n_kv_h
     if b_imp + b_rep >= L:
         return np.arange(L, dtype=np.int64), np.zeros(L, dtype=np.uint8)
     I = importance(scores32, n_kv_heads)
+    if keep_recent > 0:                      # the observation window itself is kept (SnapKV)
+        I = I.copy()
+        I[max(0, L - keep_recent):] = np.inf
     imp = top_important(I, b_imp)
     is_imp = np.zeros(L, dtype=bool)
     is_imp[imp] = True

@@ -260,3 +260,33 @@ def test_compress_sequence_end_to_end_small():
     np.testing.assert_allclose(r["colsum"].sum(axis=1), 48.0, rtol=1e-12)
     # sinks (4x key norm) receive most attention, so they are kept as important
     assert set(range(4)) <= set(r["idx"][r["kind"] == 0].tolist())
+
+
+# --- SnapKV-style pieces: pooling and the forced recent window ----------------------------------
+
+@pytest.mark.parametrize("kernel", [1, 3, 7, 13])
+def test_max_pool_matches_library_pooling(kernel):
+    s = inputs.random_scores(6, 97, 21)
+    out = O.max_pool(s, kernel)
+    ref = torch.nn.functional.max_pool1d(torch.from_numpy(s)[None], kernel, stride=1, padding=(kernel - 1) // 2)[0].numpy()
+    np.testing.assert_array_equal(out, ref)
+    assert np.all(out >= s)
+    if kernel == 1:
+        np.testing.assert_array_equal(out, s)
+
+
+def test_keep_recent_forces_the_window_into_the_important_set():
+    s = inputs.random_scores(8, 120, 23)
+    s[:, -10:] *= 1e-3                               # the recent tokens would otherwise lose
+    sig = O.signatures(s, O.thresholds(s, 30))
+    idx0, _ = O.select(s, sig, 20, 10, 8)
+    assert not set(range(110, 120)) <= set(idx0.tolist())
+    idx, kind = O.select(s, sig, 20, 10, 8, keep_recent=10)
+    assert len(idx) == 30 and set(range(110, 120)) <= set(idx[kind == 0].tolist())
+    # the other 10 important tokens are the best of the rest
+    I = O.importance(s, 8)
+    rest = sorted(sorted(range(110), key=lambda t: (-I[t], t))[:10])
+    assert sorted(set(idx[kind == 0].tolist()) - set(range(110, 120))) == rest
+    # more recent tokens than the important budget: the lowest indices of the window win the ties
+    idx2, kind2 = O.select(s, sig, 4, 3, 8, keep_recent=10)
+    assert sorted(idx2[kind2 == 0].tolist()) == [110, 111, 112, 113]
