@@ -51,9 +51,13 @@ def measured_peaks():
 # workload arithmetic (algorithmic work, independent of how the kernels do it)
 # ---------------------------------------------------------------------------------------------
 
-def algorithmic_work(w: inputs.Workload):
-    """Per step (all layers).  Causal entries per head = L(L+1)/2; 2*D flops each; two sweeps."""
-    entries = sum(L * (L + 1) // 2 if w.causal else L * L for L in w.seqlens)
+def algorithmic_work(w: inputs.Workload, window: int = 0):
+    """Per step (all layers).  Causal entries per head = L(L+1)/2 (rows of the observation window only when
+    window > 0); 2*D flops each; two sweeps."""
+    def ent(L):
+        ws = L - window if 0 < window < L else 0
+        return (L * (L + 1) // 2 - ws * (ws + 1) // 2) if w.causal else (L - ws) * L
+    entries = sum(ent(L) for L in w.seqlens)
     flops_per_sweep = 2 * w.head_dim * entries * w.n_q_heads * w.n_layers
     b_imp, b_rep = w.budgets()
     kept = int((b_imp + b_rep).sum())
@@ -271,9 +275,11 @@ def run_ours(args, w):
     kc = k if hkc is hk else hkc.to(dev, non_blocking=True)
     vc = hvc.to(dev, non_blocking=True)
     tc = vc.dtype
-    prob = B.Problem(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, causal=w.causal, device=dev)
+    prob = B.Problem(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, causal=w.causal, device=dev,
+                     query_window=args.window)
     b_imp, b_rep = w.budgets()
-    cp = B.CompressionPass(prob, b_imp[None, :], b_rep[None, :], cache_dtype=tc, impl=B.SCORE_AUTO)
+    cp = B.CompressionPass(prob, b_imp[None, :], b_rep[None, :], cache_dtype=tc, impl=B.SCORE_AUTO,
+                           pool_kernel=args.pool, keep_recent=args.window)
     torch.cuda.synchronize()
 
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
@@ -281,6 +287,8 @@ def run_ours(args, w):
     def step(marks=None):
         if marks: marks[0].record()
         cp.score(q, k)
+        if cp.pooled is not None:
+            cp.pool()
         if marks: marks[1].record()
         cp.signature()
         if marks: marks[2].record()
@@ -346,14 +354,14 @@ def run_ours(args, w):
         return
 
     peaks = measured_peaks()
-    work = algorithmic_work(w)
+    work = algorithmic_work(w, args.window)
     score_s = stage_ms[0] * 1e-3
     tensor_path = B.lib() is not None and w.qk_dtype == inputs.BF16 and w.head_dim in (64, 128)
     achieved_tf = work["score_flops"] / score_s / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
     # dram__bytes_read + dram__bytes_write of one sweep launch: 138 MB per layer in the ncu capture of a 2-layer case
     # of this workload (profiles/score_persist_kernel_cfg3_2layers.md); proportional to the layer count
-    traffic = NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP * w.n_layers if (tensor_path and w.name.startswith(DEFAULT_WORKLOAD)) else None
+    traffic = NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP * w.n_layers if (tensor_path and w.name.startswith(DEFAULT_WORKLOAD) and not args.window) else None
     roofline = {"bound": "tensor" if tensor_path else "alu", "kernel": "score_persist_kernel (two sweep launches per step; per-launch figures)" if tensor_path else "score SIMT",
                 "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
                 "traffic": traffic, "algorithmic_flops_per_launch": work["score_flops"] / 2,
@@ -386,12 +394,13 @@ def run_ours(args, w):
                    "head_dim": w.head_dim, "n_seqs": w.n_seqs, "total_tokens": w.total_tokens,
                    "budget_per_seq": [int(b_imp[0] + b_rep[0])], "cache_dtype": w.cache_dtype,
                    "l2": "inputs larger than L2 (%.1f GiB resident per step)" % (h2d / 2 ** 30),
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "query_window": args.window, "pool_kernel": args.pool},
         "layer_tokens_per_s": tokens * w.n_layers / (ms_per_step * 1e-3),
         "roofline": roofline, "stages": stages, "cpu_baseline": cpu,
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": e2e_ms},
-        "gpu_launches": 7 * args.steps,
+        "gpu_launches": (7 + (1 if cp.pooled is not None else 0)) * args.steps,
         "clocks": clocks,
     }
     print(json.dumps(line))
@@ -408,6 +417,9 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--layers", type=int, default=0, help="run only this many layers of the workload (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--window", type=int, default=0,
+                    help="SnapKV-style importance: only the last WINDOW queries vote and those tokens are kept (0 = H2O, all queries)")
+    ap.add_argument("--pool", type=int, default=0, help="max-pool the per-head scores with this odd kernel width (0 = off)")
     args = ap.parse_args()
     w = inputs.paper_workloads()[args.workload]
     if args.layers:

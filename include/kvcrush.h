@@ -89,7 +89,8 @@ typedef struct kvcrush_problem {
   int32_t max_seqlen;             /* longest sequence */
   int32_t causal;                 /* 1: query j attends keys t <= j of its own sequence; 0: all keys of the sequence */
   float   softmax_scale;          /* 0 => 1/sqrt(head_dim) (Algorithm 1) */
-  int32_t reserved;               /* set to 0 */
+  int32_t query_window;           /* 0: every query votes; w > 0: only the last w queries of each sequence
+                                     (observation window, Sec. 2.3) - kvcrush_score only */
   const int32_t* cu_seqlens_host; /* [n_seqs+1] ascending from 0; HOST copy (grid sizing) */
   const int32_t* cu_seqlens_dev;  /* the same array in device memory */
 } kvcrush_problem_t;
@@ -113,7 +114,10 @@ int kvcrush_workspace_size(const kvcrush_problem_t* problem, int stage, size_t* 
  *   scores[l][h][t] = sum over the queries j of t's sequence of A_h(j, t)
  * i.e. the attention key t receives.  (Algorithm 1 prints the sum with A_h's indices
  * in the other order, which is identically 1; the column sum is what is computed.)
- * With normalize != 0 the result is divided by the sequence length (the paper's 1/S).
+ * With normalize != 0 the result is divided by the number of voting queries (the paper's 1/S).
+ * With problem->query_window = w > 0 only the last w queries of each sequence are summed (the
+ * observation window of SnapKV, Sec. 2.3): work drops from O(S^2) to O(S*w); the row log-sum-exp
+ * is then computed (and lse_out_dev written) for those queries only.
  * The S x S matrix is never stored: a first sweep computes the log-sum-exp of every
  * query row, a second sweep recomputes the logits and accumulates exp(s - lse).
  *   Q, K        token-major tensors with n_q_heads / n_kv_heads heads, same dtype
@@ -164,6 +168,9 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
  *   anchor_mode        KVCRUSH_ANCHOR_*
  *   anchor_bits_dev    [W] uint32 (anchor_per_segment == 0) or [n_layers][n_seqs][W];
  *                      read only for KVCRUSH_ANCHOR_EXPLICIT; bits above n_q_heads ignored
+ *   keep_recent        >= 0: the last keep_recent tokens of every sequence count as infinitely
+ *                      important (the observation window is kept, as SnapKV does); they take
+ *                      places of budget_imp, lowest index first if there are more of them
  *   cu_kept_dev        [n_layers*n_seqs + 1] int32: where each segment's kept list starts
  *                      in idx_dev, segment = layer*n_seqs + seq; the caller sets it to the
  *                      prefix sums of min(budget_imp + budget_rep, length)
@@ -173,9 +180,18 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
  */
 int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
                    const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
-                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment, int keep_recent,
                    const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev,
                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * Max pooling of per-head scores along the token axis (Sec. 2.3 / 4.1.1: SnapKV keeps the
+ * neighbours of high-scoring tokens by max pooling): out[l][h][t] = max of in[l][h][t-r .. t+r]
+ * clipped to t's sequence, r = (kernel - 1) / 2.  kernel must be odd and >= 1; in and out must not
+ * alias.  Feed the result to kvcrush_signature / kvcrush_select in place of the raw scores.
+ */
+int kvcrush_pool_scores(const kvcrush_problem_t* problem, const float* scores_in_dev, int kernel,
+                        float* scores_out_dev, int32_t* status_dev, void* stream);
 
 /*
  * Stage 4 - reduced cache (Sec. 3.2: the kept tokens form the final cache).

@@ -27,7 +27,8 @@ ANCHOR_ALTERNATE, ANCHOR_MEAN, ANCHOR_EXPLICIT = 0, 1, 2
 SCORE_AUTO, SCORE_SIMT, SCORE_TENSOR = 0, 1, 2
 
 EXPORTS = ("kvcrush_workspace_size", "kvcrush_score", "kvcrush_signature", "kvcrush_select",
-           "kvcrush_compact", "kvcrush_strerror", "kvcrush_version", "kvcrush_signature_static")
+           "kvcrush_compact", "kvcrush_strerror", "kvcrush_version", "kvcrush_signature_static",
+           "kvcrush_pool_scores")
 
 
 class ProblemStruct(ctypes.Structure):
@@ -35,7 +36,7 @@ class ProblemStruct(ctypes.Structure):
         ("n_layers", ctypes.c_int32), ("n_seqs", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
         ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("total_tokens", ctypes.c_int32),
         ("max_seqlen", ctypes.c_int32), ("causal", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
-        ("reserved", ctypes.c_int32), ("cu_seqlens_host", ctypes.c_void_p), ("cu_seqlens_dev", ctypes.c_void_p),
+        ("query_window", ctypes.c_int32), ("cu_seqlens_host", ctypes.c_void_p), ("cu_seqlens_dev", ctypes.c_void_p),
     ]
 
 
@@ -68,7 +69,8 @@ def lib() -> ctypes.CDLL:
         L.kvcrush_workspace_size.argtypes = [P, i32, ctypes.POINTER(sz)]
         L.kvcrush_score.argtypes = [P, T, T, vp, vp, vp, i32, i32, vp, sz, vp, vp]
         L.kvcrush_signature.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp]
-        L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp, vp]
+        L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, i32, vp, vp, vp, vp, sz, vp, vp]
+        L.kvcrush_pool_scores.argtypes = [P, vp, i32, vp, vp, vp]
         L.kvcrush_compact.argtypes = [P, T, T, vp, vp, i64, T, T, vp, vp]
         L.kvcrush_signature_static.argtypes = [P, vp, vp, vp, vp, vp]
         L.kvcrush_strerror.argtypes = [i32]
@@ -112,7 +114,8 @@ class Problem:
     """Owns a kvcrush_problem_t plus the host and device copies of cu_seqlens it points at."""
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
-                 seqlens: Sequence[int], causal: bool = True, softmax_scale: float = 0.0, device="cuda:0"):
+                 seqlens: Sequence[int], causal: bool = True, softmax_scale: float = 0.0, device="cuda:0",
+                 query_window: int = 0):
         import torch
         self.seqlens = tuple(int(x) for x in seqlens)
         self.cu_host = np.zeros(len(self.seqlens) + 1, dtype=np.int32)
@@ -126,7 +129,7 @@ class Problem:
         self.W = (n_q_heads + 31) // 32
         self.struct = ProblemStruct(
             n_layers, self.n_seqs, n_q_heads, n_kv_heads, head_dim, self.total_tokens, self.max_seqlen,
-            int(causal), float(softmax_scale), 0, self.cu_host.ctypes.data, int(self.cu_dev.data_ptr()))
+            int(causal), float(softmax_scale), int(query_window), self.cu_host.ctypes.data, int(self.cu_dev.data_ptr()))
 
     @property
     def ref(self):
@@ -172,13 +175,19 @@ def kvcrush_signature_static(problem: Problem, scores, sigs, sig_keep, *, status
 
 
 def kvcrush_select(problem: Problem, scores, sigs, budget_imp, budget_rep, cu_kept, idx, *, kind=None,
-                   anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None, anchor_per_segment=False,
+                   anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None, anchor_per_segment=False, keep_recent=0,
                    workspace=None, status=None, stream: Optional[int] = None) -> None:
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().kvcrush_select(problem.ref, _ptr(scores), _ptr(sigs), _ptr(budget_imp), _ptr(budget_rep),
-                                int(anchor_mode), _ptr(anchor_bits), int(anchor_per_segment), _ptr(cu_kept),
+                                int(anchor_mode), _ptr(anchor_bits), int(anchor_per_segment), int(keep_recent), _ptr(cu_kept),
                                 _ptr(idx), _ptr(kind), _ptr(workspace), ws_bytes, _ptr(status),
                                 _stream() if stream is None else stream), "kvcrush_select")
+
+
+def kvcrush_pool_scores(problem: Problem, scores_in, kernel: int, scores_out, *, status=None,
+                        stream: Optional[int] = None) -> None:
+    _check(lib().kvcrush_pool_scores(problem.ref, _ptr(scores_in), int(kernel), _ptr(scores_out), _ptr(status),
+                                     _stream() if stream is None else stream), "kvcrush_pool_scores")
 
 
 def kvcrush_compact(problem: Problem, k, v, cu_kept, idx, total_kept: int, k_out, v_out, *, status=None,
@@ -202,7 +211,8 @@ class CompressionPass:
 
     def __init__(self, problem: Problem, budget_imp: np.ndarray, budget_rep: np.ndarray,
                  cache_dtype=None, sig_keep: Optional[np.ndarray] = None, anchor_mode=ANCHOR_ALTERNATE,
-                 anchor_bits: Optional[np.ndarray] = None, impl=SCORE_AUTO, with_kind=True, with_cache=True):
+                 anchor_bits: Optional[np.ndarray] = None, impl=SCORE_AUTO, with_kind=True, with_cache=True,
+                 pool_kernel: int = 0, keep_recent: int = 0):
         import torch
         p = self.problem = problem
         dev = p.device
@@ -219,14 +229,18 @@ class CompressionPass:
         keep = (bi + br) if sig_keep is None else np.broadcast_to(np.asarray(sig_keep, dtype=np.int32), (Lyr, S))
         self.budget_imp = torch.from_numpy(bi).to(dev)
         self.budget_rep = torch.from_numpy(br).to(dev)
-        self.sig_keep = torch.from_numpy(np.ascontiguousarray(keep, dtype=np.int32)).to(dev)
+        self.sig_keep = torch.from_numpy(np.array(keep, dtype=np.int32, copy=True)).to(dev)
         self.cu_kept = torch.from_numpy(self.cu_kept_host).to(dev)
         self.anchor_mode = anchor_mode
         self.anchor_bits = None if anchor_bits is None else torch.from_numpy(
             np.ascontiguousarray(anchor_bits, dtype=np.uint32).view(np.int32)).to(dev)
         self.impl = impl
+        self.pool_kernel, self.keep_recent = int(pool_kernel), int(keep_recent)
+        self.pooled = None
         self.scores = torch.empty((Lyr, p.n_q_heads, T), dtype=torch.float32, device=dev)
         self.lse = torch.empty((Lyr, p.n_q_heads, T), dtype=torch.float32, device=dev)
+        if self.pool_kernel > 1:
+            self.pooled = torch.empty((Lyr, p.n_q_heads, T), dtype=torch.float32, device=dev)
         self.theta = torch.empty((Lyr, S, p.n_q_heads), dtype=torch.float32, device=dev)
         self.sigs = torch.empty((Lyr, T, p.W), dtype=torch.int32, device=dev)
         self.idx = torch.empty((max(self.total_kept, 1),), dtype=torch.int32, device=dev)
@@ -245,14 +259,24 @@ class CompressionPass:
         kvcrush_score(self.problem, q, k, self.scores, lse_in=lse_in, lse_out=None if lse_in is not None else self.lse,
                       impl=self.impl, workspace=self.workspace, status=self.status)
 
+    def pool(self):
+        """Max-pools self.scores into self.pooled, which signature/select then use."""
+        kvcrush_pool_scores(self.problem, self.scores, self.pool_kernel, self.pooled, status=self.status)
+
+    def _selection_scores(self, scores):
+        if scores is not None:
+            return scores
+        return self.pooled if self.pooled is not None else self.scores
+
     def signature(self, scores=None):
-        kvcrush_signature(self.problem, self.scores if scores is None else scores, self.sigs,
+        kvcrush_signature(self.problem, self._selection_scores(scores), self.sigs,
                           sig_keep=self.sig_keep, theta_out=self.theta, workspace=self.workspace, status=self.status)
 
     def select(self, scores=None):
-        kvcrush_select(self.problem, self.scores if scores is None else scores, self.sigs, self.budget_imp,
+        kvcrush_select(self.problem, self._selection_scores(scores), self.sigs, self.budget_imp,
                        self.budget_rep, self.cu_kept, self.idx, kind=self.kind, anchor_mode=self.anchor_mode,
-                       anchor_bits=self.anchor_bits, workspace=self.workspace, status=self.status)
+                       anchor_bits=self.anchor_bits, keep_recent=self.keep_recent, workspace=self.workspace,
+                       status=self.status)
 
     def compact(self, k_cache, v_cache):
         kvcrush_compact(self.problem, k_cache, v_cache, self.cu_kept, self.idx, self.total_kept, self.k_out,
@@ -260,6 +284,8 @@ class CompressionPass:
 
     def run(self, q, k, k_cache=None, v_cache=None, lse_in=None):
         self.score(q, k, lse_in)
+        if self.pooled is not None:
+            self.pool()
         self.signature()
         self.select()
         if k_cache is not None:

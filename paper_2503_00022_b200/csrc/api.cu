@@ -14,7 +14,7 @@ inline size_t round_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 int make_shape(const kvcrush_problem_t* p, Shape* s) {
   if (!p) return KVCRUSH_ERR_INVALID_ARG;
   if (p->n_layers < 1 || p->n_seqs < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->head_dim < 1 ||
-      p->total_tokens < 0 || p->max_seqlen < 0)
+      p->total_tokens < 0 || p->max_seqlen < 0 || p->query_window < 0)
     return KVCRUSH_ERR_INVALID_ARG;
   if (p->n_q_heads % p->n_kv_heads != 0) return KVCRUSH_ERR_INVALID_ARG;
   if (p->n_q_heads > 128) return KVCRUSH_ERR_UNSUPPORTED;
@@ -30,6 +30,7 @@ int make_shape(const kvcrush_problem_t* p, Shape* s) {
   s->D = p->head_dim; s->T = p->total_tokens; s->max_seqlen = p->max_seqlen; s->causal = p->causal != 0;
   s->G = p->n_q_heads / p->n_kv_heads; s->W = (p->n_q_heads + 31) / 32;
   s->cu_seqlens = p->cu_seqlens_dev;
+  s->window = p->query_window;
   return KVCRUSH_OK;
 }
 
@@ -128,7 +129,7 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
 
 int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
                    const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
-                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment, int keep_recent,
                    const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev,
                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
   Shape s;
@@ -140,11 +141,12 @@ int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, co
       anchor_mode != KVCRUSH_ANCHOR_EXPLICIT)
     return KVCRUSH_ERR_INVALID_ARG;
   if (anchor_mode == KVCRUSH_ANCHOR_EXPLICIT && !anchor_bits_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if (keep_recent < 0) return KVCRUSH_ERR_INVALID_ARG;
   if (s.max_seqlen > 262144) return KVCRUSH_ERR_UNSUPPORTED;
   if (!workspace || workspace_bytes < select_workspace_bytes(s)) return KVCRUSH_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
   return launch_select(s, scores_dev, sigs_dev, budget_imp_dev, budget_rep_dev, anchor_mode, anchor_bits_dev,
-                       anchor_per_segment != 0, cu_kept_dev, idx_dev, kind_dev, workspace,
+                       anchor_per_segment != 0, keep_recent, cu_kept_dev, idx_dev, kind_dev, workspace,
                        static_cast<cudaStream_t>(stream));
 }
 
@@ -168,6 +170,16 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
   }
   return launch_compact(s, k, V ? &v : nullptr, cu_kept_dev, idx_dev, total_kept, ko, V ? &vo : nullptr,
                         static_cast<cudaStream_t>(stream));
+}
+
+int kvcrush_pool_scores(const kvcrush_problem_t* problem, const float* scores_in_dev, int kernel,
+                        float* scores_out_dev, int32_t* status_dev, void* stream) {
+  Shape s;
+  const int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if (!scores_in_dev || !scores_out_dev || !status_dev || scores_in_dev == scores_out_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if (kernel < 1 || kernel % 2 == 0) return KVCRUSH_ERR_INVALID_ARG;
+  return launch_pool_scores(s, scores_in_dev, kernel, scores_out_dev, static_cast<cudaStream_t>(stream));
 }
 
 const char* kvcrush_strerror(int code) {

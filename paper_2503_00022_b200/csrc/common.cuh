@@ -13,6 +13,7 @@ struct Shape {
   int n_layers, n_seqs, Hq, Hkv, D, T, max_seqlen, causal;
   int G;                       // Hq / Hkv
   int W;                       // signature words per token
+  int window;                  // > 0: only the last `window` queries of each sequence vote (observation window)
   const int32_t* cu_seqlens;   // device, [n_seqs + 1]
 };
 
@@ -65,7 +66,9 @@ int launch_signature(const Shape& s, const float* scores, const int32_t* sig_kee
 size_t select_workspace_bytes(const Shape& s);
 int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, const int32_t* budget_imp,
                   const int32_t* budget_rep, int anchor_mode, const uint32_t* anchor_bits, int anchor_per_segment,
-                  const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws, cudaStream_t stream);
+                  int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws, cudaStream_t stream);
+
+int launch_pool_scores(const Shape& s, const float* scores_in, int kernel, float* scores_out, cudaStream_t stream);
 
 int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, const int32_t* cu_kept,
                    const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,

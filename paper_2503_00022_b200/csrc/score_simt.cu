@@ -76,6 +76,8 @@ lse_rows_kernel(Shape s, TensorView Q, TensorView K, float scale_log2, float* __
   const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
   const int t0 = __ldg(s.cu_seqlens + seq), t1 = __ldg(s.cu_seqlens + seq + 1);
   const int t_end = s.causal ? tok + 1 : t1;
+  const int ws = (s.window > 0 && t1 - t0 > s.window) ? t1 - t0 - s.window : 0;   // first voting query of the sequence
+  if (tok - t0 < ws) return;                       // this query does not vote: its log-sum-exp is not needed
 
   const T* q = static_cast<const T*>(Q.ptr) + layer * Q.sl + (long long)tok * Q.st + h * Q.sh;
   const T* kbase = static_cast<const T*>(K.ptr) + layer * K.sl + (h / s.G) * K.sh;
@@ -112,7 +114,8 @@ colsum_kernel(Shape s, TensorView Q, TensorView K, float scale_log2, const float
   const int layer = (int)(col / ((long long)s.T * s.Hq));
   const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
   const int t0 = __ldg(s.cu_seqlens + seq), t1 = __ldg(s.cu_seqlens + seq + 1);
-  const int j_begin = s.causal ? tok : t0;
+  const int ws = (s.window > 0 && t1 - t0 > s.window) ? t1 - t0 - s.window : 0;   // first voting query of the sequence
+  const int j_begin = max(s.causal ? tok : t0, t0 + ws);
 
   const T* k = static_cast<const T*>(K.ptr) + layer * K.sl + (long long)tok * K.st + (h / s.G) * K.sh;
   const T* qbase = static_cast<const T*>(Q.ptr) + layer * Q.sl + h * Q.sh;
@@ -126,7 +129,7 @@ colsum_kernel(Shape s, TensorView Q, TensorView K, float scale_log2, const float
   }
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, d);
-  if (lane == 0) scores[col] = normalize ? acc / (float)(t1 - t0) : acc;
+  if (lane == 0) scores[col] = normalize ? acc / (float)(t1 - t0 - ws) : acc;
 }
 
 template <typename T>

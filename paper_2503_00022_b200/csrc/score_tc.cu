@@ -90,6 +90,7 @@ struct PAux {
 template <bool kColsum>
 struct Geo {
   int layer, h, hk, t0, L, blk, first_stream, n_iter;
+  int ws;                      // first query row that votes (0 without an observation window)
   bool causal, half1;
   __device__ __forceinline__ Geo(const Shape& s, const int* it) {
     layer = it[0]; h = it[1]; hk = h / s.G; blk = it[3];
@@ -98,8 +99,9 @@ struct Geo {
     L = __ldg(s.cu_seqlens + seq + 1) - t0;
     causal = s.causal != 0;
     half1 = blk * kBlockRows + kTile < L;                               // does the second half hold any row
+    ws = (s.window > 0 && L > s.window) ? L - s.window : 0;
     if (kColsum) {                                                      // stationary keys, streamed query tiles
-      first_stream = causal ? 2 * blk : 0;
+      first_stream = max(causal ? 2 * blk : 0, ws / kTile);
       n_iter = n_tiles - first_stream;
     } else {                                                            // stationary queries, streamed key tiles
       first_stream = 0;
@@ -110,10 +112,10 @@ struct Geo {
   __device__ __forceinline__ bool active(int hf, int it) const {
     if (hf == 1 && !half1) return false;
     if (!causal) return true;
-    return kColsum ? it >= hf : it <= 2 * blk + hf;
+    return kColsum ? first_stream + it >= 2 * blk + hf : it <= 2 * blk + hf;
   }
   __device__ __forceinline__ bool diag(int hf, int it) const {
-    return causal && (kColsum ? it == hf : it == 2 * blk + hf);
+    return causal && (kColsum ? first_stream + it == 2 * blk + hf : it == 2 * blk + hf);
   }
 };
 
@@ -189,7 +191,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       const int lh = idx / a.n_items, rank = idx - lh * a.n_items;
       int seq, blk, nblk;
-      decode_item(s.cu_seqlens, s.n_seqs, a.max_blocks, rank, !kColsum, lane, seq, blk, nblk, kBlockRows);
+      decode_item(s.cu_seqlens, s.n_seqs, a.max_blocks, rank, !kColsum, lane, seq, blk, nblk, kBlockRows, s.window);
       if (lane == 0) {
         int* it = aux->item[slot];
         it[0] = lh / s.Hq; it[1] = lh - it[0] * s.Hq; it[2] = seq; it[3] = blk;
@@ -332,11 +334,11 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const float* lse_row = a.lse + ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0;
         auto load_lse = [&](int i) {                // minus lse2 of this thread's query of streamed tile i (-inf past the end)
           const int j = (g.first_stream + i) * kTile + r;
-          return (i < g.n_iter && j < g.L) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
+          return (i < g.n_iter && j < g.L && j >= g.ws) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
         };
         f32x2 acc[2] = {0ull, 0ull};
         // this group's tiles of the item: every other active tile, starting where the running parity says
-        int first = g.causal ? hf : 0;
+        int first = g.causal ? max(0, 2 * g.blk + hf - g.first_stream) : 0;
         if (((cnt & 1) != par)) ++first;
         float lse_next = load_lse(first);
         int n_mine = 0;
@@ -368,7 +370,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (!ok) break;
         if (par == 0 && row < g.L && (hf == 0 || g.half1)) {
           total += part[r];
-          if (a.normalize) total = total / (float)g.L;
+          if (a.normalize) total = total / (float)(g.L - g.ws);
           a.scores[out] = total;
         }
       } else {
@@ -398,7 +400,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         pair_sync();
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
-        if (par == 0 && row < g.L && (hf == 0 || g.half1)) {       // merge the other group's (max, sum)
+        if (par == 0 && row < g.L && row >= g.ws && (hf == 0 || g.half1)) {   // merge the other group's (max, sum)
           const float m1 = pm[r], sum1 = ps[r];
           const float big = fmaxf(m, m1);
           const float tot = (sum > 0.f ? sum * ex2(m - big) : 0.f) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
@@ -458,17 +460,23 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
   PersistArgs a{};
   a.s = s; a.scale_log2 = scale_log2; a.normalize = normalize; a.status = status; a.scores = scores;
   a.max_blocks = (s.max_seqlen + kBlockRows - 1) / kBlockRows;
-  long long items = 0;
-  for (int i = 0; i < s.n_seqs; ++i) items += (cu_host[i + 1] - cu_host[i] + kBlockRows - 1) / kBlockRows;
-  if (items == 0) return KVCRUSH_OK;
-  const long long total = items * s.n_layers * s.Hq;
-  if (total > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
-  a.n_items = (int)items;
-  a.total_items = (int)total;
+  // work items per (layer, head): every 256-row block for the column sweep; for the row sweep only the
+  // blocks that hold voting queries
+  long long items_col = 0, items_row = 0;
+  for (int i = 0; i < s.n_seqs; ++i) {
+    const int len = cu_host[i + 1] - cu_host[i];
+    const int nb = (len + kBlockRows - 1) / kBlockRows;
+    const int first = (s.window > 0 && len > s.window) ? (len - s.window) / kBlockRows : 0;
+    items_col += nb;
+    items_row += nb - first;
+  }
+  if (items_col == 0) return KVCRUSH_OK;
+  if (items_col * s.n_layers * s.Hq > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
   if (cudaMemsetAsync(counters, 0, 2 * sizeof(int), stream) != cudaSuccess) return KVCRUSH_ERR_CUDA;
   int rc;
   if (!lse_in) {
     a.lse2_out = lse2_ws; a.lse_nat_out = lse_out; a.counter = counters;
+    a.n_items = (int)items_row; a.total_items = (int)(items_row * s.n_layers * s.Hq);
     rc = s.D == 128 ? launch_persist<128, false>(mq, mk, a, n_sms, stream) : launch_persist<64, false>(mq, mk, a, n_sms, stream);
     if (rc != KVCRUSH_OK) return rc;
     a.lse = lse2_ws; a.lse_mul = 1.f;
@@ -476,6 +484,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
     a.lse = lse_in; a.lse_mul = lse_in_mul;
   }
   a.counter = counters + 1;
+  a.n_items = (int)items_col; a.total_items = (int)(items_col * s.n_layers * s.Hq);
   return s.D == 128 ? launch_persist<128, true>(mq, mk, a, n_sms, stream) : launch_persist<64, true>(mq, mk, a, n_sms, stream);
 }
 

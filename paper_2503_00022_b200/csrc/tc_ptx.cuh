@@ -295,22 +295,28 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
 // Items are (sequence, tile) pairs; an item's weight w is the number of 128x128 tiles it sweeps
 // (causal: query tile q sweeps q+1 key tiles; key tile k sweeps n-k query tiles).  Rank j counts items
 // in order of decreasing w, sequences in order inside one w.  Runs on one full warp.
+// With an observation window (window > 0) a row sweep only has the items that hold one of the last
+// `window` rows of their sequence; `tile` is then still the item's index inside the whole sequence.
 __device__ __forceinline__ void decode_item(const int32_t* __restrict__ cu, int n_seqs, int max_tiles, int j,
                                             bool row_sweep, int lane, int& seq, int& tile, int& n_tiles,
-                                            int rows_per_item = 128) {
+                                            int rows_per_item, int window) {
   int rem = j;
   seq = 0; tile = 0; n_tiles = 0;
   for (int w = max_tiles; w >= 1; --w) {
     for (int base = 0; base < n_seqs; base += 32) {
       const int s = base + lane;
-      const int nt = s < n_seqs ? (__ldg(cu + s + 1) - __ldg(cu + s) + rows_per_item - 1) / rows_per_item : 0;
-      const unsigned mask = __ballot_sync(0xFFFFFFFFu, nt >= w);
+      const int len = s < n_seqs ? __ldg(cu + s + 1) - __ldg(cu + s) : 0;
+      const int nt = (len + rows_per_item - 1) / rows_per_item;
+      const int first = (row_sweep && window > 0 && len > window) ? (len - window) / rows_per_item : 0;
+      const int cnt_s = nt - first;
+      const unsigned mask = __ballot_sync(0xFFFFFFFFu, cnt_s >= w);
       const int cnt = __popc(mask);
       if (rem < cnt) {
         const int pos = __fns(mask, 0, rem + 1);
         seq = base + pos;
         n_tiles = __shfl_sync(0xFFFFFFFFu, nt, pos);
-        tile = row_sweep ? w - 1 : n_tiles - w;
+        const int first_p = __shfl_sync(0xFFFFFFFFu, first, pos);
+        tile = row_sweep ? first_p + w - 1 : n_tiles - w;
         return;
       }
       rem -= cnt;

@@ -38,7 +38,7 @@ def test_library_exports_every_declared_symbol(lib):
 def _problem(**over):
     cu = np.asarray(over.pop("cu", [0, 100]), dtype=np.int32)
     kw = dict(n_layers=1, n_seqs=len(cu) - 1, n_q_heads=8, n_kv_heads=4, head_dim=64, total_tokens=int(cu[-1]),
-              max_seqlen=int(np.diff(cu).max()), causal=1, softmax_scale=0.0, reserved=0,
+              max_seqlen=int(np.diff(cu).max()), causal=1, softmax_scale=0.0, query_window=0,
               cu_seqlens_host=cu.ctypes.data, cu_seqlens_dev=0x1000)
     kw.update(over)
     p = B.ProblemStruct(**kw)
@@ -57,7 +57,7 @@ def test_workspace_sizes_and_shape_validation(lib):
     assert lib.kvcrush_workspace_size(ctypes.byref(p), 9, ctypes.byref(out)) == B.ERR_INVALID_ARG
     assert lib.kvcrush_workspace_size(None, 0, ctypes.byref(out)) == B.ERR_INVALID_ARG
     for bad in (dict(n_kv_heads=3), dict(n_layers=0), dict(total_tokens=99), dict(max_seqlen=50),
-                dict(cu_seqlens_dev=None), dict(cu=[0, 60, 40])):
+                dict(cu_seqlens_dev=None), dict(cu=[0, 60, 40]), dict(query_window=-1)):
         q = _problem(**bad)
         assert lib.kvcrush_workspace_size(ctypes.byref(q), 0, ctypes.byref(out)) == B.ERR_INVALID_ARG, bad
     assert lib.kvcrush_workspace_size(ctypes.byref(_problem(n_q_heads=256, n_kv_heads=256)), 0,
@@ -81,12 +81,17 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
     assert lib.kvcrush_signature(r(p), 0x100, None, None, 0x100, None, None, 0, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_signature(r(p), 0x100, 0x100, None, 0x100, None, None, 0, 0x100, None) == B.ERR_WORKSPACE
     # select: anchor mode range, explicit anchor needs bits, workspace
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 5, None, 0, 0x100, 0x100, None, 0x100, 1 << 20,
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 5, None, 0, 0, 0x100, 0x100, None, 0x100, 1 << 20,
                               0x100, None) == B.ERR_INVALID_ARG
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, B.ANCHOR_EXPLICIT, None, 0, 0x100, 0x100, None,
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, B.ANCHOR_EXPLICIT, None, 0, 0, 0x100, 0x100, None,
                               0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, 0x100, 0x100, None, 0x100, 16,
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, 0, 0x100, 0x100, None, 0x100, 16,
                               0x100, None) == B.ERR_WORKSPACE
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, -1, 0x100, 0x100, None, 0x100, 1 << 20,
+                              0x100, None) == B.ERR_INVALID_ARG
+    # pooling: even kernel, aliasing
+    assert lib.kvcrush_pool_scores(r(p), 0x100, 4, 0x200, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_pool_scores(r(p), 0x100, 3, 0x100, 0x100, None) == B.ERR_INVALID_ARG
     # compact: V without V_out, dtype mismatch, negative count
     assert lib.kvcrush_compact(r(p), r(t), r(t), 0x100, 0x100, 10, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_compact(r(p), r(t), None, 0x100, 0x100, 10, r(f16), None, 0x100, None) == B.ERR_INVALID_ARG
