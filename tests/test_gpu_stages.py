@@ -278,3 +278,26 @@ def test_score_head_major_layout_and_explicit_scale(B, impl_name):
             a, b = int(cu[s_]), int(cu[s_ + 1])
             c, _ = O.scores(inputs.widen(li.q[a:b], w.qk_dtype), inputs.widen(li.k[a:b], w.qk_dtype), True, scale=scale)
             assert TL.within_score_tolerance(g[l][:, a:b], c).all()
+
+
+def test_score_leaves_at_once_when_status_already_flags_an_error(B):
+    """The tensor-core kernels read the status word first: a launch that follows a reported device error does
+    no work (outputs untouched) and keeps the first error's record."""
+    import torch
+    dev = _dev()
+    w = TENSOR_CASES[1]
+    lis, q, k, _, _ = TL.stack_layers(w, range(1), with_cache=False)
+    prob = B.Problem(1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, device=dev)
+    scores = torch.full((1, w.n_q_heads, w.total_tokens), -5.0, dtype=torch.float32, device=dev)
+    ws = torch.empty(B.kvcrush_workspace_size(prob, B.STAGE_SCORE), dtype=torch.uint8, device=dev)
+    status = torch.tensor([B.DEV_TIMEOUT, 2, 17, 0], dtype=torch.int32, device=dev)
+    B.kvcrush_score(prob, TL.torch_storage(q, w.qk_dtype, dev), TL.torch_storage(k, w.qk_dtype, dev), scores,
+                    impl=B.SCORE_TENSOR, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [B.DEV_TIMEOUT, 2, 17, 0]
+    assert bool((scores == -5.0).all())
+    status.zero_()                                           # and the same call works once the word is cleared
+    B.kvcrush_score(prob, TL.torch_storage(q, w.qk_dtype, dev), TL.torch_storage(k, w.qk_dtype, dev), scores,
+                    impl=B.SCORE_TENSOR, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0 and bool((scores >= 0).all())
