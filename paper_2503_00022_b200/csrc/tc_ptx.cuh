@@ -302,6 +302,12 @@ __device__ __forceinline__ void decode_item(const int32_t* __restrict__ cu, int 
                                             int rows_per_item, int window) {
   int rem = j;
   seq = 0; tile = 0; n_tiles = 0;
+  if (n_seqs == 1) {                               // one sequence: rank j is simply the j-th heaviest item
+    const int len = __ldg(cu + 1) - __ldg(cu);
+    n_tiles = (len + rows_per_item - 1) / rows_per_item;
+    tile = row_sweep ? n_tiles - 1 - j : j;
+    return;
+  }
   for (int w = max_tiles; w >= 1; --w) {
     for (int base = 0; base < n_seqs; base += 32) {
       const int s = base + lane;
