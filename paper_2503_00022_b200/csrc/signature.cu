@@ -44,6 +44,15 @@ theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __
   const float* row = scores + ((size_t)layer * s.Hq + h) * s.T + t0;
   const int lane = threadIdx.x & 31;
 
+  // When the row fits, its order keys are first copied into shared memory with independent, coalesced loads
+  // (the sweeps below interleave every load with warp votes and atomics, which would expose the full global
+  // latency once per element).
+  if (stage_row) {
+#pragma unroll 4
+    for (int i = threadIdx.x; i < L; i += kSelectThreads) row_keys[i] = order_key(__ldg(row + i));
+    __syncthreads();
+  }
+
   uint32_t prefix = 0;       // selected high digits so far
   uint32_t k_rem = keep;     // rank among the elements that share the prefix
   for (int shift = 24; shift >= 0; shift -= 8) {
@@ -53,15 +62,7 @@ theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __
     for (int base = 0; base < L; base += kSelectThreads) {
       const int i = base + threadIdx.x;
       const bool in = i < L;
-      // the first sweep reads the scores and, when the row fits, leaves its keys in shared memory for the other three
-      uint32_t key = 0u;
-      if (in) {
-        if (stage_row && shift != 24) key = row_keys[i];
-        else {
-          key = order_key(__ldg(row + i));
-          if (stage_row) row_keys[i] = key;
-        }
-      }
+      const uint32_t key = !in ? 0u : stage_row ? row_keys[i] : order_key(__ldg(row + i));
       const bool live = in && ((key & hi_mask) == prefix);
       const uint32_t digit = (key >> shift) & 0xFFu;
       // high digits (sign, exponent) are the same for almost every score: one add per warp then;
