@@ -54,6 +54,14 @@ because it gives no formula for them:
   width (positions outside the sequence do not count);
 * ``select(..., keep_recent=n)``: the last n tokens are important by decree (their
   importance is +inf) and count against B_important.
+
+Chunk- and page-granular eviction (Sec. 4.3.4: chunks of 8 tokens; Sec. 4.3.5: pages of 32 tokens): the
+paper gives two sentences - the baseline sums the attention weights over a page, and the
+binary vector of a page is the concatenation of the head vectors of its tokens.  Everything
+else follows the token-level steps with a page in the place of a token
+(``page_importance``, ``page_vectors``, ``select_pages``, ``compact_pages``).  PARITY UNPINNED:
+a short last page counts its missing tokens as all-zero vectors of zero importance, and the
+anchor of a page repeats the token anchor once per slot.
 """
 from __future__ import annotations
 
@@ -344,6 +352,80 @@ def select(scores32: np.ndarray, sig: np.ndarray, b_imp: int, b_rep: int, n_kv_h
     kind = np.zeros(kept.shape[0], dtype=np.uint8)
     kind[np.isin(kept, reps)] = 1
     return kept, kind
+
+
+# ---------------------------------------------------------------------------
+# Page / chunk granularity (Sec. 4.3.4, Sec. 4.3.5)
+# ---------------------------------------------------------------------------
+
+def page_importance(I: np.ndarray, page_size: int) -> np.ndarray:
+    """Importance of page p = sum of I(t) over its tokens, float64, added one token at a
+    time in ascending order (Sec. 4.3.5: the baseline aggregates the attention sums per page)."""
+    L = I.shape[0]
+    n_pages = (L + page_size - 1) // page_size
+    J = np.zeros(n_pages, dtype=np.float64)
+    for i in range(page_size):
+        t = np.arange(n_pages) * page_size + i
+        ok = t < L
+        J[ok] = J[ok] + I[t[ok]]
+    return J
+
+
+def page_vectors(sig: np.ndarray, page_size: int) -> np.ndarray:
+    """Binary vector of a page = its tokens' head vectors one after the other (Sec. 4.3.5):
+    uint32 [n_pages, page_size * W]; slots past the end of the sequence are zero."""
+    L, W = sig.shape
+    n_pages = (L + page_size - 1) // page_size
+    out = np.zeros((n_pages * page_size, W), dtype=np.uint32)
+    out[:L] = sig
+    return out.reshape(n_pages, page_size * W)
+
+
+def select_pages(scores32: np.ndarray, sig: np.ndarray, page_size: int, b_imp: int, b_rep: int,
+                 n_kv_heads: int, anchor_mode: int = ANCHOR_ALTERNATE,
+                 explicit_anchor: Optional[np.ndarray] = None):
+    """Kept page ids (ascending) and their kind; budgets count pages.  The steps are those of
+    ``select`` with pages for tokens: page importance, top b_imp pages, then Algorithm 2 on the
+    page vectors of the other pages."""
+    Hq, L = scores32.shape
+    W = sig.shape[1]
+    n_pages = (L + page_size - 1) // page_size
+    if b_imp + b_rep >= n_pages:
+        return np.arange(n_pages, dtype=np.int64), np.zeros(n_pages, dtype=np.uint8)
+    J = page_importance(importance(scores32, n_kv_heads), page_size)
+    imp = top_important(J, b_imp)
+    is_imp = np.zeros(n_pages, dtype=bool)
+    is_imp[imp] = True
+    reps = np.zeros(0, dtype=np.int64)
+    if b_rep > 0:
+        n_bits = 32 * page_size * W              # unused bits of every word are zero on both sides
+        vec = page_vectors(sig & _head_mask(Hq)[None, :], page_size)
+        cand = np.nonzero(~is_imp)[0]
+        N = cand.shape[0]
+        if anchor_mode == ANCHOR_MEAN:
+            a = anchor_bits(ANCHOR_MEAN, n_bits, vec[cand])
+        else:
+            a = np.tile(anchor_bits(anchor_mode, Hq, None, explicit_anchor), page_size)
+        d = hamming(vec[cand], a, n_bits)
+        srt = cand[np.lexsort((cand, d))]
+        bounds = bucket_bounds(N, b_rep)
+        reps = np.asarray([representative(srt[bounds[i]:bounds[i + 1]], vec[srt[bounds[i]:bounds[i + 1]]], n_bits)
+                           for i in range(b_rep)], dtype=np.int64)
+    kept = np.sort(np.concatenate([imp, reps]))
+    kind = np.zeros(kept.shape[0], dtype=np.uint8)
+    kind[np.isin(kept, reps)] = 1
+    return kept, kind
+
+
+def compact_pages(cache: np.ndarray, page_idx: np.ndarray, page_size: int) -> np.ndarray:
+    """Reduced paged cache [n_kept, page_size, ...]: the kept pages of a token-major cache
+    [L, ...]; the slots of a short last page are zero."""
+    L = cache.shape[0]
+    out = np.zeros((len(page_idx), page_size) + cache.shape[1:], dtype=cache.dtype)
+    for i, p in enumerate(np.asarray(page_idx, dtype=np.int64)):
+        n = min(page_size, L - int(p) * page_size)
+        out[i, :n] = cache[int(p) * page_size:int(p) * page_size + n]
+    return out
 
 
 def compact(cache: np.ndarray, idx: np.ndarray) -> np.ndarray:
