@@ -209,6 +209,46 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
                     int32_t* status_dev, void* stream);
 
 /*
+ * Stage 3 at page (or chunk) granularity (Sec. 4.3.4: chunks of 8 tokens; Sec. 4.3.5: pages of 32 tokens, where
+ * the baseline sums the attention weights over a page and the binary vector of a page is the concatenation of the
+ * head vectors of its tokens).  A page is page_size consecutive tokens of one sequence, page p = tokens
+ * [p*page_size, (p+1)*page_size); the last page may be short: its missing tokens count as all-zero vectors of zero
+ * importance.  Budgets, cu_kept and the output count PAGES.
+ *   J(p)  = sum of I(t) over the tokens of p (I as in kvcrush_select), float64, tokens in ascending order
+ *   Imp   = the budget_imp pages of largest J (ties: lower page)
+ *   v_p   = sigs of the page's tokens one after the other (page_size * W words); anchor: the token anchor in
+ *           every slot (ALTERNATE, EXPLICIT) or the per-bit majority of the grouped pages (MEAN, ties to 1)
+ *   then exactly the steps of kvcrush_select on the other pages: d_p = popcount(v_p xor anchor), (d_p, p) order,
+ *   budget_rep equal-frequency buckets, per bucket the page closest to the per-bit mean (L1; ties: lower page),
+ *   kept = Imp U representatives, ascending.  budget_imp + budget_rep >= number of pages keeps every page.
+ *   page_size          >= 1; page_size * W <= 128 words and at most 8192 pages per sequence, otherwise
+ *                      KVCRUSH_ERR_UNSUPPORTED.  page_size 1 gives the result of kvcrush_select (keep_recent 0).
+ *   anchor_bits_dev    [W] or [n_layers][n_seqs][W] token anchor (EXPLICIT only)
+ *   cu_kept_dev        [n_layers*n_seqs + 1] prefix sums of min(budget_imp + budget_rep, pages of the sequence)
+ *   page_idx_dev       out [cu_kept[last]] int32 page number inside its sequence
+ *   kind_dev           optional out: 0 important, 1 representative
+ *   workspace          kvcrush_workspace_size(.., KVCRUSH_STAGE_SELECT, ..) bytes
+ */
+int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
+                         int page_size, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+                         int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                         const int32_t* cu_kept_dev, int32_t* page_idx_dev, uint8_t* kind_dev,
+                         void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * Stage 4 at page granularity (Sec. 4.3.5): the kept pages form the reduced paged cache.
+ *   out[l][(cu_kept[l*n_seqs+s] - cu_kept[l*n_seqs] + i) * page_size + j][h][:] =
+ *        in[l][cu_seqlens[s] + page_idx[cu_kept[l*n_seqs+s] + i] * page_size + j][h][:]     j < page_size
+ *   and zeros for the slots j of a short last page that lie past the end of the sequence.
+ *   total_kept_pages   cu_kept[n_layers*n_seqs] (host value)
+ * Other arguments as for kvcrush_compact; the outputs hold total kept pages * page_size token rows per layer.
+ */
+int kvcrush_compact_pages(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K, const kvcrush_tensor_t* V,
+                          int page_size, const int32_t* cu_kept_dev, const int32_t* page_idx_dev,
+                          int64_t total_kept_pages, const kvcrush_tensor_t* K_out, const kvcrush_tensor_t* V_out,
+                          int32_t* status_dev, void* stream);
+
+/*
  * Stage 2 without caller-provided scratch (the paper has no counterpart; this is a packaging
  * variant of kvcrush_signature for hosts that cannot hand over device memory).
  *

@@ -28,7 +28,7 @@ SCORE_AUTO, SCORE_SIMT, SCORE_TENSOR = 0, 1, 2
 
 EXPORTS = ("kvcrush_workspace_size", "kvcrush_score", "kvcrush_signature", "kvcrush_select",
            "kvcrush_compact", "kvcrush_strerror", "kvcrush_version", "kvcrush_signature_static",
-           "kvcrush_pool_scores")
+           "kvcrush_pool_scores", "kvcrush_select_pages", "kvcrush_compact_pages")
 
 
 class ProblemStruct(ctypes.Structure):
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, i32, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_pool_scores.argtypes = [P, vp, i32, vp, vp, vp]
         L.kvcrush_compact.argtypes = [P, T, T, vp, vp, i64, T, T, vp, vp]
+        L.kvcrush_select_pages.argtypes = [P, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp, vp]
+        L.kvcrush_compact_pages.argtypes = [P, T, T, i32, vp, vp, i64, T, T, vp, vp]
         L.kvcrush_signature_static.argtypes = [P, vp, vp, vp, vp, vp]
         L.kvcrush_strerror.argtypes = [i32]
         L.kvcrush_strerror.restype = ctypes.c_char_p
@@ -201,32 +203,59 @@ def kvcrush_compact(problem: Problem, k, v, cu_kept, idx, total_kept: int, k_out
                                  _stream() if stream is None else stream), "kvcrush_compact")
 
 
+def kvcrush_select_pages(problem: Problem, scores, sigs, page_size: int, budget_imp, budget_rep, cu_kept, page_idx, *,
+                         kind=None, anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None, anchor_per_segment=False,
+                         workspace=None, status=None, stream: Optional[int] = None) -> None:
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().kvcrush_select_pages(problem.ref, _ptr(scores), _ptr(sigs), int(page_size), _ptr(budget_imp),
+                                      _ptr(budget_rep), int(anchor_mode), _ptr(anchor_bits), int(anchor_per_segment),
+                                      _ptr(cu_kept), _ptr(page_idx), _ptr(kind), _ptr(workspace), ws_bytes,
+                                      _ptr(status), _stream() if stream is None else stream), "kvcrush_select_pages")
+
+
+def kvcrush_compact_pages(problem: Problem, k, v, page_size: int, cu_kept, page_idx, total_kept_pages: int, k_out,
+                          v_out, *, status=None, stream: Optional[int] = None) -> None:
+    ks, kos = tensor_struct(k), tensor_struct(k_out)
+    vs = tensor_struct(v) if v is not None else None
+    vos = tensor_struct(v_out) if v_out is not None else None
+    _check(lib().kvcrush_compact_pages(problem.ref, ctypes.byref(ks), ctypes.byref(vs) if vs is not None else None,
+                                       int(page_size), _ptr(cu_kept), _ptr(page_idx), int(total_kept_pages),
+                                       ctypes.byref(kos), ctypes.byref(vos) if vos is not None else None,
+                                       _ptr(status), _stream() if stream is None else stream), "kvcrush_compact_pages")
+
+
 class CompressionPass:
     """All buffers of one compression pass, allocated once; ``run`` enqueues the four stages.
 
     q [Lyr, T, Hq, D], k [Lyr, T, Hkv, D] (scoring inputs) and the K/V caches are the caller's
     tensors; budgets are per (layer, sequence) numpy arrays.  Nothing here computes: it
     sizes and allocates outputs and workspaces and forwards pointers.
+
+    page_size > 0 selects and gathers whole pages of that many tokens: budgets then count pages,
+    ``idx`` holds page numbers and the reduced cache has page_size rows per kept page.
     """
 
     def __init__(self, problem: Problem, budget_imp: np.ndarray, budget_rep: np.ndarray,
                  cache_dtype=None, sig_keep: Optional[np.ndarray] = None, anchor_mode=ANCHOR_ALTERNATE,
                  anchor_bits: Optional[np.ndarray] = None, impl=SCORE_AUTO, with_kind=True, with_cache=True,
-                 pool_kernel: int = 0, keep_recent: int = 0):
+                 pool_kernel: int = 0, keep_recent: int = 0, page_size: int = 0):
         import torch
+        self.page_size = int(page_size)
+        assert not (self.page_size and keep_recent), "keep_recent is a token-level option"
+        unit = max(self.page_size, 1)
         p = self.problem = problem
         dev = p.device
         Lyr, S, T = p.n_layers, p.n_seqs, p.total_tokens
         bi = np.broadcast_to(np.asarray(budget_imp, dtype=np.int32), (Lyr, S)).copy()
         br = np.broadcast_to(np.asarray(budget_rep, dtype=np.int32), (Lyr, S)).copy()
-        lens = np.asarray(p.seqlens, dtype=np.int64)[None, :]
+        lens = (np.asarray(p.seqlens, dtype=np.int64)[None, :] + unit - 1) // unit       # tokens, or pages
         kept = np.minimum(bi.astype(np.int64) + br, lens)
         cu_kept = np.zeros(Lyr * S + 1, dtype=np.int64)
         cu_kept[1:] = np.cumsum(kept.reshape(-1))
         self.kept_per_layer = kept.sum(axis=1)
         self.total_kept = int(cu_kept[-1])
         self.cu_kept_host = cu_kept.astype(np.int32)
-        keep = (bi + br) if sig_keep is None else np.broadcast_to(np.asarray(sig_keep, dtype=np.int32), (Lyr, S))
+        keep = (bi + br) * unit if sig_keep is None else np.broadcast_to(np.asarray(sig_keep, dtype=np.int32), (Lyr, S))
         self.budget_imp = torch.from_numpy(bi).to(dev)
         self.budget_rep = torch.from_numpy(br).to(dev)
         self.sig_keep = torch.from_numpy(np.array(keep, dtype=np.int32, copy=True)).to(dev)
@@ -250,7 +279,7 @@ class CompressionPass:
         self.workspace = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=dev)
         self.k_out = self.v_out = None
         if with_cache and cache_dtype is not None:
-            n_out = int(self.kept_per_layer.max()) if Lyr else 0
+            n_out = int(self.kept_per_layer.max()) * unit if Lyr else 0
             shape = (Lyr, max(n_out, 1), p.n_kv_heads, p.head_dim)
             self.k_out = torch.empty(shape, dtype=cache_dtype, device=dev)
             self.v_out = torch.empty(shape, dtype=cache_dtype, device=dev)
@@ -273,12 +302,22 @@ class CompressionPass:
                           sig_keep=self.sig_keep, theta_out=self.theta, workspace=self.workspace, status=self.status)
 
     def select(self, scores=None):
+        if self.page_size:
+            kvcrush_select_pages(self.problem, self._selection_scores(scores), self.sigs, self.page_size,
+                                 self.budget_imp, self.budget_rep, self.cu_kept, self.idx, kind=self.kind,
+                                 anchor_mode=self.anchor_mode, anchor_bits=self.anchor_bits,
+                                 workspace=self.workspace, status=self.status)
+            return
         kvcrush_select(self.problem, self._selection_scores(scores), self.sigs, self.budget_imp,
                        self.budget_rep, self.cu_kept, self.idx, kind=self.kind, anchor_mode=self.anchor_mode,
                        anchor_bits=self.anchor_bits, keep_recent=self.keep_recent, workspace=self.workspace,
                        status=self.status)
 
     def compact(self, k_cache, v_cache):
+        if self.page_size:
+            kvcrush_compact_pages(self.problem, k_cache, v_cache, self.page_size, self.cu_kept, self.idx,
+                                  self.total_kept, self.k_out, self.v_out, status=self.status)
+            return
         kvcrush_compact(self.problem, k_cache, v_cache, self.cu_kept, self.idx, self.total_kept, self.k_out,
                         self.v_out, status=self.status)
 
@@ -297,7 +336,7 @@ class CompressionPass:
             raise RuntimeError(f"kvcrush device error {st}")
 
     def kept(self, layer: int, seq: int) -> np.ndarray:
-        """Kept token ids (host copy) of one (layer, sequence)."""
+        """Kept token ids (page numbers when page_size > 0; host copy) of one (layer, sequence)."""
         seg = layer * self.problem.n_seqs + seq
         lo, hi = int(self.cu_kept_host[seg]), int(self.cu_kept_host[seg + 1])
         return self.idx[lo:hi].cpu().numpy()

@@ -172,6 +172,53 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
                         static_cast<cudaStream_t>(stream));
 }
 
+int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
+                         int page_size, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+                         int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                         const int32_t* cu_kept_dev, int32_t* page_idx_dev, uint8_t* kind_dev,
+                         void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  Shape s;
+  const int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if (!scores_dev || !sigs_dev || !budget_imp_dev || !budget_rep_dev || !cu_kept_dev || !page_idx_dev || !status_dev)
+    return KVCRUSH_ERR_INVALID_ARG;
+  if (anchor_mode != KVCRUSH_ANCHOR_ALTERNATE && anchor_mode != KVCRUSH_ANCHOR_MEAN &&
+      anchor_mode != KVCRUSH_ANCHOR_EXPLICIT)
+    return KVCRUSH_ERR_INVALID_ARG;
+  if (anchor_mode == KVCRUSH_ANCHOR_EXPLICIT && !anchor_bits_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if (page_size < 1) return KVCRUSH_ERR_INVALID_ARG;
+  if ((long long)page_size * s.W > kMaxPageWords) return KVCRUSH_ERR_UNSUPPORTED;
+  if (((long long)s.max_seqlen + page_size - 1) / page_size > kMaxPagesPerSeq) return KVCRUSH_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < select_workspace_bytes(s)) return KVCRUSH_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
+  return launch_select_pages(s, scores_dev, sigs_dev, page_size, budget_imp_dev, budget_rep_dev, anchor_mode,
+                             anchor_bits_dev, anchor_per_segment != 0, cu_kept_dev, page_idx_dev, kind_dev,
+                             workspace, static_cast<cudaStream_t>(stream));
+}
+
+int kvcrush_compact_pages(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K, const kvcrush_tensor_t* V,
+                          int page_size, const int32_t* cu_kept_dev, const int32_t* page_idx_dev,
+                          int64_t total_kept_pages, const kvcrush_tensor_t* K_out, const kvcrush_tensor_t* V_out,
+                          int32_t* status_dev, void* stream) {
+  Shape s;
+  int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if (!cu_kept_dev || !page_idx_dev || !status_dev || total_kept_pages < 0 || page_size < 1)
+    return KVCRUSH_ERR_INVALID_ARG;
+  if ((V == nullptr) != (V_out == nullptr)) return KVCRUSH_ERR_INVALID_ARG;
+  TensorView k, v, ko, vo;
+  if ((rc = make_view(K, s.D, &k)) != KVCRUSH_OK) return rc;
+  if ((rc = make_view(K_out, s.D, &ko)) != KVCRUSH_OK) return rc;
+  if (k.dtype != ko.dtype) return KVCRUSH_ERR_INVALID_ARG;
+  if (V) {
+    if ((rc = make_view(V, s.D, &v)) != KVCRUSH_OK) return rc;
+    if ((rc = make_view(V_out, s.D, &vo)) != KVCRUSH_OK) return rc;
+    if (v.dtype != k.dtype || vo.dtype != k.dtype) return KVCRUSH_ERR_INVALID_ARG;
+  }
+  return launch_compact_pages(s, k, V ? &v : nullptr, page_size, cu_kept_dev, page_idx_dev, total_kept_pages, ko,
+                              V ? &vo : nullptr, static_cast<cudaStream_t>(stream));
+}
+
 int kvcrush_pool_scores(const kvcrush_problem_t* problem, const float* scores_in_dev, int kernel,
                         float* scores_out_dev, int32_t* status_dev, void* stream) {
   Shape s;

@@ -5,6 +5,9 @@
 // copies that token's rows of every KV head, for K and for V, as 16-byte vectors: the index
 // arithmetic (segment search, source token) is paid once per token, and every lane keeps four
 // independent 16-byte loads in flight before the first store.
+//
+// Page-granular variant (Sec. 4.3.5: paged caches keep or drop whole pages): the kept list holds page numbers,
+// a warp owns one token slot of one kept page, and the slots of a short last page are filled with zeros.
 #include "common.cuh"
 
 namespace kvc {
@@ -23,11 +26,15 @@ struct CompactArgs {
   int n_vec;                                   // vectors per token = Hkv * vec_per_row
 };
 
+template <bool kPaged>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 compact_kernel(Shape s, CompactArgs a, const int32_t* __restrict__ cu_kept, const int32_t* __restrict__ idx,
-               long long total_kept) {
+               long long total_kept, int page_size) {
   const int lane = threadIdx.x & 31;
-  const long long row = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  const long long out_row = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  // row = position in the kept list (a token, or a page of which this warp copies slot `slot`)
+  const long long row = kPaged ? out_row / page_size : out_row;
+  const int slot = kPaged ? (int)(out_row - row * page_size) : 0;
   if (row >= total_kept) return;
 
   // segment = layer * n_seqs + seq that owns kept row `row`
@@ -38,8 +45,18 @@ compact_kernel(Shape s, CompactArgs a, const int32_t* __restrict__ cu_kept, cons
     if ((long long)__ldg(cu_kept + mid) <= row) lo = mid; else hi = mid;
   }
   const int layer = lo / s.n_seqs, seq = lo - layer * s.n_seqs;
-  const long long src_tok = (long long)__ldg(s.cu_seqlens + seq) + __ldg(idx + row);
-  const long long dst_tok = row - __ldg(cu_kept + layer * s.n_seqs);
+  long long src_tok, dst_tok;
+  bool present = true;
+  if (kPaged) {
+    const long long tok_in_seq = (long long)__ldg(idx + row) * page_size + slot;
+    const int seq_begin = __ldg(s.cu_seqlens + seq);
+    present = tok_in_seq < __ldg(s.cu_seqlens + seq + 1) - seq_begin;
+    src_tok = seq_begin + tok_in_seq;
+    dst_tok = (row - __ldg(cu_kept + layer * s.n_seqs)) * page_size + slot;
+  } else {
+    src_tok = (long long)__ldg(s.cu_seqlens + seq) + __ldg(idx + row);
+    dst_tok = row - __ldg(cu_kept + layer * s.n_seqs);
+  }
 
 #pragma unroll 1
   for (int ten = 0; ten < a.n_tensors; ++ten) {
@@ -50,7 +67,8 @@ compact_kernel(Shape s, CompactArgs a, const int32_t* __restrict__ cu_kept, cons
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int v = v0 + u * 32;
-        if (v < a.n_vec) {
+        if (kPaged) val[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (v < a.n_vec && (!kPaged || present)) {
           const int h = v / a.vec_per_row, c = v - h * a.vec_per_row;
           val[u] = __ldcs(reinterpret_cast<const uint4*>(sp + h * a.src_sh[ten]) + c);
         }
@@ -69,9 +87,11 @@ compact_kernel(Shape s, CompactArgs a, const int32_t* __restrict__ cu_kept, cons
 
 }  // namespace
 
-int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, const int32_t* cu_kept,
-                   const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,
-                   cudaStream_t stream) {
+namespace {
+
+int launch_gather(const Shape& s, const TensorView& K, const TensorView* V, int page_size, const int32_t* cu_kept,
+                  const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,
+                  cudaStream_t stream) {
   if (total_kept == 0) return KVCRUSH_OK;
   const int eb = elt_bytes(K.dtype);
   CompactArgs a{};
@@ -86,10 +106,28 @@ int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, con
   }
   a.vec_per_row = s.D * eb / 16;
   a.n_vec = s.Hkv * a.vec_per_row;
-  const long long blocks = (total_kept + kWarpsPerBlock - 1) / kWarpsPerBlock;
+  const long long rows = total_kept * (page_size > 0 ? page_size : 1);
+  const long long blocks = (rows + kWarpsPerBlock - 1) / kWarpsPerBlock;
   if (blocks > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
-  compact_kernel<<<(unsigned)blocks, kWarpsPerBlock * 32, 0, stream>>>(s, a, cu_kept, idx, total_kept);
+  if (page_size > 0)
+    compact_kernel<true><<<(unsigned)blocks, kWarpsPerBlock * 32, 0, stream>>>(s, a, cu_kept, idx, total_kept, page_size);
+  else
+    compact_kernel<false><<<(unsigned)blocks, kWarpsPerBlock * 32, 0, stream>>>(s, a, cu_kept, idx, total_kept, 1);
   return check_launch();
+}
+
+}  // namespace
+
+int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, const int32_t* cu_kept,
+                   const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,
+                   cudaStream_t stream) {
+  return launch_gather(s, K, V, 0, cu_kept, idx, total_kept, K_out, V_out, stream);
+}
+
+int launch_compact_pages(const Shape& s, const TensorView& K, const TensorView* V, int page_size,
+                         const int32_t* cu_kept, const int32_t* page_idx, long long total_kept_pages,
+                         const TensorView& K_out, const TensorView* V_out, cudaStream_t stream) {
+  return launch_gather(s, K, V, page_size, cu_kept, page_idx, total_kept_pages, K_out, V_out, stream);
 }
 
 }  // namespace kvc

@@ -15,16 +15,17 @@
 //                               per-bit mean, up to a constant), ties to the lower token
 //                            5. kept = important U representatives, ascending token index
 // All decisions are integer or exact float64 comparisons, so the result is unique.
-#include "common.cuh"
+#include "select_common.cuh"
 
 namespace kvc {
 
 namespace {
 
-constexpr int kThreads = 1024;
-constexpr int kWarps = kThreads / 32;
+using sel::kThreads;
+using sel::kWarps;
+using sel::kFull;
+using sel::head_mask;
 constexpr int kMaxBins = 129;              // Hamming distances 0..128
-constexpr unsigned kFull = 0xFFFFFFFFu;
 
 __global__ void __launch_bounds__(256)
 importance_kernel(Shape s, const float* __restrict__ scores, int keep_recent, unsigned long long* __restrict__ keys) {
@@ -74,11 +75,6 @@ struct SelectArgs {
   int stage_sorted, stage_sig, stage_keys;   // which per-segment arrays are copied into shared memory
 };
 
-__device__ __forceinline__ uint32_t head_mask(int Hq, int w) {
-  const int n = Hq - 32 * w;
-  return n >= 32 ? 0xFFFFFFFFu : ((1u << n) - 1u);
-}
-
 template <int W>                       // signature words per token (compile time: the per-word loops unroll)
 __global__ void __launch_bounds__(kThreads, 1)
 select_segment_kernel(Shape s, SelectArgs a) {
@@ -86,12 +82,9 @@ select_segment_kernel(Shape s, SelectArgs a) {
   uint32_t* imp_mask = dyn_smem;
   uint32_t* rep_mask = dyn_smem + a.mask_words;
 
-  __shared__ uint32_t hist[256];
-  __shared__ unsigned long long sel_prefix;
-  __shared__ uint32_t sel_k;
+  __shared__ sel::Scratch sc;
   __shared__ int warp_hist[kWarps][kMaxBins];
   __shared__ int bin_base[kMaxBins + 1];
-  __shared__ int warp_tot[kWarps];
   __shared__ int bit_cnt[128];
   __shared__ uint32_t anchor_sh[4];
 
@@ -135,91 +128,14 @@ select_segment_kernel(Shape s, SelectArgs a) {
     }
   }
   const int n_words = (L + 31) >> 5;
-  // contiguous token range of this warp (multiple of 32 tokens so that mask words do not straddle)
-  const int per_warp = ((n_words + kWarps - 1) / kWarps) * 32;
-  const int r_lo = min(L, warp * per_warp), r_hi = min(L, r_lo + per_warp);
+  int r_lo, r_hi;                            // contiguous token range of this warp
+  sel::warp_range(L, warp, r_lo, r_hi);
 
   for (int i = tid; i < n_words; i += kThreads) { imp_mask[i] = 0; rep_mask[i] = 0; }
   __syncthreads();
 
   // ---- 1. important tokens: the b_imp largest keys, ties to the lower index --------------------
-  if (b_imp > 0) {
-    unsigned long long prefix = 0;
-    uint32_t k_rem = b_imp;
-    for (int shift = 56; shift >= 0; shift -= 8) {
-      for (int i = tid; i < 256; i += kThreads) hist[i] = 0;
-      __syncthreads();
-      const unsigned long long hi_mask = shift == 56 ? 0ull : (~0ull << (shift + 8));
-      for (int base = 0; base < L; base += kThreads) {
-        const int i = base + tid;
-        const bool in = i < L;
-        const unsigned long long key = in ? keys[i] : 0ull;
-        const bool live = in && ((key & hi_mask) == prefix);
-        const uint32_t digit = (uint32_t)(key >> shift) & 0xFFu;
-        // high digits (sign, exponent) are the same for almost every key: one add per warp then;
-        // low digits are spread over the 256 bins, where plain shared-memory atomics do not collide much
-        const unsigned voters = __ballot_sync(kFull, live);
-        if (voters) {
-          const uint32_t d0 = __shfl_sync(kFull, digit, __ffs(voters) - 1);
-          if (__all_sync(kFull, !live || digit == d0)) {
-            if (lane == 0) atomicAdd(&hist[d0], __popc(voters));
-          } else if (live) {
-            atomicAdd(&hist[digit], 1u);
-          }
-        }
-      }
-      __syncthreads();
-      if (warp == 0) {
-        uint32_t local = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) local += hist[255 - 8 * lane - j];
-        uint32_t incl = local;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          const uint32_t v = __shfl_up_sync(kFull, incl, d);
-          if (lane >= d) incl += v;
-        }
-        const uint32_t excl = incl - local;
-        if (excl < k_rem && k_rem <= incl) {
-          uint32_t acc = excl;
-          for (int j = 0; j < 8; ++j) {
-            const uint32_t c = hist[255 - 8 * lane - j];
-            if (k_rem <= acc + c) {
-              sel_prefix = prefix | ((unsigned long long)(255 - 8 * lane - j) << shift);
-              sel_k = k_rem - acc;
-              break;
-            }
-            acc += c;
-          }
-        }
-      }
-      __syncthreads();
-      prefix = sel_prefix;
-      k_rem = sel_k;
-      __syncthreads();
-    }
-    // prefix = the b_imp-th largest key; k_rem = how many keys equal to it are admitted
-    const unsigned long long kth = prefix;
-    int n_eq = 0;
-    for (int i = r_lo + lane; i < r_hi; i += 32) n_eq += (keys[i] == kth);
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) n_eq += __shfl_xor_sync(kFull, n_eq, d);
-    if (lane == 0) warp_tot[warp] = n_eq;
-    __syncthreads();
-    int eq_before = 0;
-    for (int w = 0; w < warp; ++w) eq_before += warp_tot[w];
-    for (int base = r_lo; base < r_hi; base += 32) {
-      const int i = base + lane;
-      const unsigned long long key = i < r_hi ? keys[i] : 0ull;
-      const bool eq = i < r_hi && key == kth;
-      const unsigned eq_b = __ballot_sync(kFull, eq);
-      const bool imp = i < r_hi && (key > kth || (eq && (uint32_t)(eq_before + __popc(eq_b & lt_mask)) < k_rem));
-      const unsigned imp_b = __ballot_sync(kFull, imp);
-      if (lane == 0) imp_mask[base >> 5] = imp_b;
-      eq_before += __popc(eq_b);
-    }
-    __syncthreads();
-  }
+  if (b_imp > 0) sel::mark_top_keys(keys, L, b_imp, imp_mask, sc);
 
   // ---- 2-4. representatives of the other tokens ------------------------------------------------
   if (b_rep > 0) {
@@ -384,35 +300,17 @@ select_segment_kernel(Shape s, SelectArgs a) {
   }
 
   // ---- 5. kept = important U representatives, ascending ------------------------------------------
-  const int wpt = (n_words + kThreads - 1) / kThreads;      // mask words per thread, contiguous
-  const int w_lo = min(n_words, tid * wpt), w_hi = min(n_words, w_lo + wpt);
-  int cnt = 0;
-  for (int w = w_lo; w < w_hi; ++w) cnt += __popc(imp_mask[w] | rep_mask[w]);
-  int incl = cnt;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const int v = __shfl_up_sync(kFull, incl, d);
-    if (lane >= d) incl += v;
-  }
-  __syncthreads();                          // warp_tot is reused
-  if (lane == 31) warp_tot[warp] = incl;
-  __syncthreads();
-  int pos = incl - cnt;
-  for (int w = 0; w < warp; ++w) pos += warp_tot[w];
-  for (int w = w_lo; w < w_hi; ++w) {
-    const uint32_t rep = rep_mask[w];
-    uint32_t bits = imp_mask[w] | rep;
-    while (bits) {
-      const int b = __ffs(bits) - 1;
-      bits &= bits - 1;
-      out_idx[pos] = 32 * w + b;
-      if (out_kind) out_kind[pos] = (rep >> b) & 1u;
-      ++pos;
-    }
-  }
+  sel::emit_kept(imp_mask, rep_mask, n_words, out_idx, out_kind, sc);
 }
 
 }  // namespace
+
+int launch_importance(const Shape& s, const float* scores, int keep_recent, unsigned long long* keys,
+                      cudaStream_t stream) {
+  const size_t n = (size_t)s.n_layers * s.T;
+  importance_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, scores, keep_recent, keys);
+  return check_launch();
+}
 
 size_t select_workspace_bytes(const Shape& s) {
   const size_t n = (size_t)s.n_layers * s.T;
@@ -426,8 +324,7 @@ int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, con
   const size_t n = (size_t)s.n_layers * s.T;
   unsigned long long* keys = static_cast<unsigned long long*>(ws);
   int32_t* sorted = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(ws) + ((n * 8 + 255) / 256) * 256);
-  importance_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, scores, keep_recent, keys);
-  if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+  if (launch_importance(s, scores, keep_recent, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
 
   SelectArgs a{};
   a.keys = keys; a.sigs = sigs; a.budget_imp = budget_imp; a.budget_rep = budget_rep;

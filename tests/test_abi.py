@@ -89,6 +89,16 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
                               0x100, None) == B.ERR_WORKSPACE
     assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, -1, 0x100, 0x100, None, 0x100, 1 << 20,
                               0x100, None) == B.ERR_INVALID_ARG
+    # page-granular select: page size, page vector too long, too many pages per sequence, workspace
+    sp = lambda ps, prob=p, ws=1 << 20: lib.kvcrush_select_pages(r(prob), 0x100, 0x100, ps, 0x100, 0x100, 0, None, 0, 0x100,
+                                                                 0x100, None, 0x100, ws, 0x100, None)
+    assert sp(0) == B.ERR_INVALID_ARG
+    assert sp(256) == B.ERR_UNSUPPORTED
+    assert sp(8, ws=16) == B.ERR_WORKSPACE
+    long_seq = _problem(cu=[0, 100000])
+    assert sp(8, prob=long_seq, ws=1 << 30) == B.ERR_UNSUPPORTED
+    assert lib.kvcrush_compact_pages(r(p), r(t), None, 0, 0x100, 0x100, 10, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_compact_pages(r(p), r(t), r(t), 8, 0x100, 0x100, 10, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
     # pooling: even kernel, aliasing
     assert lib.kvcrush_pool_scores(r(p), 0x100, 4, 0x200, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_pool_scores(r(p), 0x100, 3, 0x100, 0x100, None) == B.ERR_INVALID_ARG
