@@ -278,8 +278,12 @@ def run_ours(args, w):
     prob = B.Problem(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, causal=w.causal, device=dev,
                      query_window=args.window)
     b_imp, b_rep = w.budgets()
+    if args.page_size:                                    # page-granular eviction: the same token budget, in whole pages
+        pages = np.maximum((b_imp + b_rep) // args.page_size, 1)
+        b_rep = (pages // 2).astype(np.int32)
+        b_imp = (pages - b_rep).astype(np.int32)
     cp = B.CompressionPass(prob, b_imp[None, :], b_rep[None, :], cache_dtype=tc, impl=B.SCORE_AUTO,
-                           pool_kernel=args.pool, keep_recent=args.window)
+                           pool_kernel=args.pool, keep_recent=args.window, page_size=args.page_size)
     torch.cuda.synchronize()
 
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
@@ -355,7 +359,7 @@ def run_ours(args, w):
         pr = B.Problem(nl, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, causal=w.causal, device=dev,
                        query_window=args.window)
         passes.append(B.CompressionPass(pr, b_imp[None, :], b_rep[None, :], cache_dtype=tc, impl=B.SCORE_AUTO,
-                                        pool_kernel=args.pool, keep_recent=args.window))
+                                        pool_kernel=args.pool, keep_recent=args.window, page_size=args.page_size))
     equal_chunks = all(bounds[c + 1] - bounds[c] == bounds[1] - bounds[0] for c in range(n_chunks))
     h_idx = [torch.empty(passes[0].idx.shape, dtype=torch.int32, pin_memory=True) for _ in range(n_chunks)]
     h_ko = [torch.empty(passes[0].k_out.shape, dtype=tc, pin_memory=True) for _ in range(n_chunks)]
@@ -416,6 +420,9 @@ def run_ours(args, w):
 
     peaks = measured_peaks()
     work = algorithmic_work(w, args.window)
+    if args.page_size:                                    # rows actually gathered: kept pages x page size
+        eb = inputs.storage_itemsize(w.cache_dtype)
+        work["compact_bytes"] = 2 * 2 * cp.total_kept * args.page_size * w.n_kv_heads * w.head_dim * eb
     score_s = stage_ms[0] * 1e-3
     tensor_path = B.lib() is not None and w.qk_dtype == inputs.BF16 and w.head_dim in (64, 128)
     achieved_tf = work["score_flops"] / score_s / 1e12
@@ -458,7 +465,7 @@ def run_ours(args, w):
                    "budget_per_seq": [int(b_imp[0] + b_rep[0])], "cache_dtype": w.cache_dtype,
                    "l2": "inputs larger than L2 (%.1f GiB resident per step)" % (h2d / 2 ** 30),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "query_window": args.window, "pool_kernel": args.pool},
+                   "query_window": args.window, "pool_kernel": args.pool, "page_size": args.page_size},
         "layer_tokens_per_s": tokens * w.n_layers / (ms_per_step * 1e-3),
         "roofline": roofline, "stages": stages, "cpu_baseline": cpu,
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -486,7 +493,11 @@ def main():
     ap.add_argument("--window", type=int, default=0,
                     help="SnapKV-style importance: only the last WINDOW queries vote and those tokens are kept (0 = H2O, all queries)")
     ap.add_argument("--pool", type=int, default=0, help="max-pool the per-head scores with this odd kernel width (0 = off)")
+    ap.add_argument("--page-size", type=int, default=0,
+                    help="evict whole pages of this many tokens (8 = the paper's chunks, 32 = its pages; 0 = token level)")
     args = ap.parse_args()
+    if args.page_size and args.window:
+        ap.error("--page-size and --window are separate modes")
     w = inputs.paper_workloads()[args.workload]
     if args.layers:
         w = inputs.shrink(w, args.layers)

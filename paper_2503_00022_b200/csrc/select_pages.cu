@@ -92,7 +92,14 @@ select_pages_kernel(Shape s, PageArgs a) {
   for (int p = tid; p < n_pages; p += kThreads) {
     const int first = p * P, n_tok = min(P, L - first);
     double acc = 0.0;
-    for (int i = 0; i < n_tok; ++i) acc = __dadd_rn(acc, key_to_double(tkeys[first + i]));
+    for (int i0 = 0; i0 < n_tok; i0 += 8) {        // the adds are sequential by definition, the loads are not
+      unsigned long long kk[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) kk[j] = i0 + j < n_tok ? tkeys[first + i0 + j] : 0ull;
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (i0 + j < n_tok) acc = __dadd_rn(acc, key_to_double(kk[j]));
+    }
     pkeys[p] = double_to_key(acc);
   }
   for (int i = tid; i < n_words; i += kThreads) { imp_mask[i] = 0; rep_mask[i] = 0; }
