@@ -53,7 +53,9 @@ because it gives no formula for them:
 * ``max_pool``: every per-head score becomes the maximum over a centred window of odd
   width (positions outside the sequence do not count);
 * ``select(..., keep_recent=n)``: the last n tokens are important by decree (their
-  importance is +inf) and count against B_important.
+  importance is +inf) and count against B_important; ``keep_initial=n`` does the same for
+  the first n tokens (Table 1 splits its 672-token budget into 32 initial + 512 middle +
+  128 recent tokens).
 
 Chunk- and page-granular eviction (Sec. 4.3.4: chunks of 8 tokens; Sec. 4.3.5: pages of 32 tokens): the
 paper gives two sentences - the baseline sums the attention weights over a page, and the
@@ -323,17 +325,19 @@ def representative(member_tokens: np.ndarray, member_sigs: np.ndarray, n_q_heads
 
 def select(scores32: np.ndarray, sig: np.ndarray, b_imp: int, b_rep: int, n_kv_heads: int,
            anchor_mode: int = ANCHOR_ALTERNATE, explicit_anchor: Optional[np.ndarray] = None,
-           keep_recent: int = 0):
+           keep_recent: int = 0, keep_initial: int = 0):
     """Kept token ids (ascending) and their kind (0 important, 1 representative).
 
-    A budget b_imp + b_rep >= L keeps every token (kind 0)."""
+    A budget b_imp + b_rep >= L keeps every token (kind 0).  The first keep_initial and the last
+    keep_recent tokens are important by decree (Table 1: initial and recent parts of the budget)."""
     Hq, L = scores32.shape
     if b_imp + b_rep >= L:
         return np.arange(L, dtype=np.int64), np.zeros(L, dtype=np.uint8)
     I = importance(scores32, n_kv_heads)
-    if keep_recent > 0:                      # the observation window itself is kept (SnapKV)
+    if keep_recent > 0 or keep_initial > 0:  # the observation window (SnapKV) / the attention sinks are kept
         I = I.copy()
         I[max(0, L - keep_recent):] = np.inf
+        I[:min(L, keep_initial)] = np.inf
     imp = top_important(I, b_imp)
     is_imp = np.zeros(L, dtype=bool)
     is_imp[imp] = True
@@ -383,16 +387,18 @@ def page_vectors(sig: np.ndarray, page_size: int) -> np.ndarray:
 
 def select_pages(scores32: np.ndarray, sig: np.ndarray, page_size: int, b_imp: int, b_rep: int,
                  n_kv_heads: int, anchor_mode: int = ANCHOR_ALTERNATE,
-                 explicit_anchor: Optional[np.ndarray] = None):
+                 explicit_anchor: Optional[np.ndarray] = None, keep_recent: int = 0, keep_initial: int = 0):
     """Kept page ids (ascending) and their kind; budgets count pages.  The steps are those of
     ``select`` with pages for tokens: page importance, top b_imp pages, then Algorithm 2 on the
-    page vectors of the other pages."""
+    page vectors of the other pages.  keep_initial / keep_recent count pages too."""
     Hq, L = scores32.shape
     W = sig.shape[1]
     n_pages = (L + page_size - 1) // page_size
     if b_imp + b_rep >= n_pages:
         return np.arange(n_pages, dtype=np.int64), np.zeros(n_pages, dtype=np.uint8)
     J = page_importance(importance(scores32, n_kv_heads), page_size)
+    J[max(0, n_pages - keep_recent):] = np.inf
+    J[:min(n_pages, keep_initial)] = np.inf
     imp = top_important(J, b_imp)
     is_imp = np.zeros(n_pages, dtype=bool)
     is_imp[imp] = True

@@ -160,3 +160,28 @@ def test_compact_pages_is_a_padded_library_gather():
     got = O.compact_pages(cache, pages, P)
     assert got.tobytes() == want.tobytes()
     assert not got[2, 5:].any()                            # slots past the end of the sequence
+
+
+def test_paged_budget_of_table1_keeps_initial_and_recent_pages():
+    """Table 1's paged setting: 672 tokens = 32 initial + 512 middle + 128 recent at page size 32, i.e. 1 + 16 + 4
+    pages, a quarter of the middle pages chosen as representatives."""
+    P, L, Hq = 32, 4000, 8
+    s = inputs.random_scores(Hq, L, 51)
+    s[:, :P] *= 1e-3
+    s[:, -4 * P:] *= 1e-3
+    sig = _sigs_for(s, 672)
+    idx, kind = O.select_pages(s, sig, P, 17, 4, 8, keep_initial=1, keep_recent=4)
+    n_pages = (L + P - 1) // P
+    assert len(idx) == 21
+    forced = {0} | set(range(n_pages - 4, n_pages))
+    assert forced <= set(idx[kind == 0].tolist())
+    J = O.page_importance(O.importance(s, 8), P)
+    middle = sorted(sorted(set(range(n_pages)) - forced, key=lambda p: (-J[p], p))[:12])
+    assert sorted(set(idx[kind == 0].tolist()) - forced) == middle
+    # same thing through raised scores and no decree
+    raised = s.copy()
+    raised[:, :P] = 1e6
+    raised[:, (n_pages - 4) * P:] = 1e6
+    want = O.select_pages(raised, sig, P, 17, 4, 8)
+    np.testing.assert_array_equal(idx, want[0])
+    np.testing.assert_array_equal(kind, want[1])

@@ -290,3 +290,23 @@ def test_keep_recent_forces_the_window_into_the_important_set():
     # more recent tokens than the important budget: the lowest indices of the window win the ties
     idx2, kind2 = O.select(s, sig, 4, 3, 8, keep_recent=10)
     assert sorted(idx2[kind2 == 0].tolist()) == [110, 111, 112, 113]
+
+
+def test_keep_initial_and_recent_equal_selection_on_raised_scores():
+    """Tokens kept by decree behave like tokens whose scores beat everything: the pinned routine run on
+    scores with those columns raised (signatures unchanged) gives the same kept set."""
+    s = inputs.random_scores(8, 150, 29, tie_levels=2)
+    s[:, :6] *= 1e-3                                  # the initial tokens would otherwise lose
+    sig = O.signatures(s, O.thresholds(s, 40))
+    raised = s.copy()
+    raised[:, :6] = 1e6
+    raised[:, -9:] = 1e6
+    for b_imp, b_rep in ((25, 15), (15, 25), (40, 0)):
+        want = O.select(raised, sig, b_imp, b_rep, 4)
+        got = O.select(s, sig, b_imp, b_rep, 4, keep_recent=9, keep_initial=6)
+        np.testing.assert_array_equal(got[0], want[0])
+        np.testing.assert_array_equal(got[1], want[1])
+        assert set(range(6)) | set(range(141, 150)) <= set(got[0][got[1] == 0].tolist())
+    # more forced tokens than places: the lowest indices win (initial tokens first)
+    idx, kind = O.select(s, sig, 8, 4, 4, keep_recent=9, keep_initial=6)
+    assert sorted(idx[kind == 0].tolist()) == [0, 1, 2, 3, 4, 5, 141, 142]
