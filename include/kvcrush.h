@@ -168,9 +168,10 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
  *   anchor_mode        KVCRUSH_ANCHOR_*
  *   anchor_bits_dev    [W] uint32 (anchor_per_segment == 0) or [n_layers][n_seqs][W];
  *                      read only for KVCRUSH_ANCHOR_EXPLICIT; bits above n_q_heads ignored
- *   keep_recent        >= 0: the last keep_recent tokens of every sequence count as infinitely
- *                      important (the observation window is kept, as SnapKV does); they take
- *                      places of budget_imp, lowest index first if there are more of them
+ *   keep_initial,      >= 0: the first keep_initial and the last keep_recent tokens of every sequence count
+ *   keep_recent        as infinitely important (Table 1 of the paper reserves initial and recent parts of the
+ *                      budget; SnapKV keeps its observation window); they take places of budget_imp,
+ *                      lowest index first if there are more of them
  *   cu_kept_dev        [n_layers*n_seqs + 1] int32: where each segment's kept list starts
  *                      in idx_dev, segment = layer*n_seqs + seq; the caller sets it to the
  *                      prefix sums of min(budget_imp + budget_rep, length)
@@ -180,7 +181,8 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
  */
 int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
                    const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
-                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment, int keep_recent,
+                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                   int keep_initial, int keep_recent,
                    const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev,
                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
@@ -222,8 +224,10 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
  *   budget_rep equal-frequency buckets, per bucket the page closest to the per-bit mean (L1; ties: lower page),
  *   kept = Imp U representatives, ascending.  budget_imp + budget_rep >= number of pages keeps every page.
  *   page_size          >= 1; page_size * W <= 128 words and at most 8192 pages per sequence, otherwise
- *                      KVCRUSH_ERR_UNSUPPORTED.  page_size 1 gives the result of kvcrush_select (keep_recent 0).
+ *                      KVCRUSH_ERR_UNSUPPORTED.  page_size 1 gives the result of kvcrush_select.
  *   anchor_bits_dev    [W] or [n_layers][n_seqs][W] token anchor (EXPLICIT only)
+ *   keep_initial,      >= 0, in pages: the first / last pages of every sequence are important by decree (Table 1:
+ *   keep_recent        a 672-token budget = 32 initial + 512 middle + 128 recent tokens at page size 32)
  *   cu_kept_dev        [n_layers*n_seqs + 1] prefix sums of min(budget_imp + budget_rep, pages of the sequence)
  *   page_idx_dev       out [cu_kept[last]] int32 page number inside its sequence
  *   kind_dev           optional out: 0 important, 1 representative
@@ -232,6 +236,7 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
 int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
                          int page_size, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
                          int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                         int keep_initial, int keep_recent,
                          const int32_t* cu_kept_dev, int32_t* page_idx_dev, uint8_t* kind_dev,
                          void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 

@@ -69,10 +69,10 @@ def lib() -> ctypes.CDLL:
         L.kvcrush_workspace_size.argtypes = [P, i32, ctypes.POINTER(sz)]
         L.kvcrush_score.argtypes = [P, T, T, vp, vp, vp, i32, i32, vp, sz, vp, vp]
         L.kvcrush_signature.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp]
-        L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, i32, vp, vp, vp, vp, sz, vp, vp]
+        L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_pool_scores.argtypes = [P, vp, i32, vp, vp, vp]
         L.kvcrush_compact.argtypes = [P, T, T, vp, vp, i64, T, T, vp, vp]
-        L.kvcrush_select_pages.argtypes = [P, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp, vp]
+        L.kvcrush_select_pages.argtypes = [P, vp, vp, i32, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_compact_pages.argtypes = [P, T, T, i32, vp, vp, i64, T, T, vp, vp]
         L.kvcrush_signature_static.argtypes = [P, vp, vp, vp, vp, vp]
         L.kvcrush_strerror.argtypes = [i32]
@@ -178,10 +178,11 @@ def kvcrush_signature_static(problem: Problem, scores, sigs, sig_keep, *, status
 
 def kvcrush_select(problem: Problem, scores, sigs, budget_imp, budget_rep, cu_kept, idx, *, kind=None,
                    anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None, anchor_per_segment=False, keep_recent=0,
-                   workspace=None, status=None, stream: Optional[int] = None) -> None:
+                   keep_initial=0, workspace=None, status=None, stream: Optional[int] = None) -> None:
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().kvcrush_select(problem.ref, _ptr(scores), _ptr(sigs), _ptr(budget_imp), _ptr(budget_rep),
-                                int(anchor_mode), _ptr(anchor_bits), int(anchor_per_segment), int(keep_recent), _ptr(cu_kept),
+                                int(anchor_mode), _ptr(anchor_bits), int(anchor_per_segment), int(keep_initial),
+                                int(keep_recent), _ptr(cu_kept),
                                 _ptr(idx), _ptr(kind), _ptr(workspace), ws_bytes, _ptr(status),
                                 _stream() if stream is None else stream), "kvcrush_select")
 
@@ -205,11 +206,12 @@ def kvcrush_compact(problem: Problem, k, v, cu_kept, idx, total_kept: int, k_out
 
 def kvcrush_select_pages(problem: Problem, scores, sigs, page_size: int, budget_imp, budget_rep, cu_kept, page_idx, *,
                          kind=None, anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None, anchor_per_segment=False,
-                         workspace=None, status=None, stream: Optional[int] = None) -> None:
+                         keep_initial=0, keep_recent=0, workspace=None, status=None,
+                         stream: Optional[int] = None) -> None:
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().kvcrush_select_pages(problem.ref, _ptr(scores), _ptr(sigs), int(page_size), _ptr(budget_imp),
                                       _ptr(budget_rep), int(anchor_mode), _ptr(anchor_bits), int(anchor_per_segment),
-                                      _ptr(cu_kept), _ptr(page_idx), _ptr(kind), _ptr(workspace), ws_bytes,
+                                      int(keep_initial), int(keep_recent), _ptr(cu_kept), _ptr(page_idx), _ptr(kind), _ptr(workspace), ws_bytes,
                                       _ptr(status), _stream() if stream is None else stream), "kvcrush_select_pages")
 
 
@@ -232,16 +234,16 @@ class CompressionPass:
     sizes and allocates outputs and workspaces and forwards pointers.
 
     page_size > 0 selects and gathers whole pages of that many tokens: budgets then count pages,
-    ``idx`` holds page numbers and the reduced cache has page_size rows per kept page.
+    ``idx`` holds page numbers, the reduced cache has page_size rows per kept page and keep_initial /
+    keep_recent count pages as well.
     """
 
     def __init__(self, problem: Problem, budget_imp: np.ndarray, budget_rep: np.ndarray,
                  cache_dtype=None, sig_keep: Optional[np.ndarray] = None, anchor_mode=ANCHOR_ALTERNATE,
                  anchor_bits: Optional[np.ndarray] = None, impl=SCORE_AUTO, with_kind=True, with_cache=True,
-                 pool_kernel: int = 0, keep_recent: int = 0, page_size: int = 0):
+                 pool_kernel: int = 0, keep_recent: int = 0, page_size: int = 0, keep_initial: int = 0):
         import torch
         self.page_size = int(page_size)
-        assert not (self.page_size and keep_recent), "keep_recent is a token-level option"
         unit = max(self.page_size, 1)
         p = self.problem = problem
         dev = p.device
@@ -264,7 +266,7 @@ class CompressionPass:
         self.anchor_bits = None if anchor_bits is None else torch.from_numpy(
             np.ascontiguousarray(anchor_bits, dtype=np.uint32).view(np.int32)).to(dev)
         self.impl = impl
-        self.pool_kernel, self.keep_recent = int(pool_kernel), int(keep_recent)
+        self.pool_kernel, self.keep_recent, self.keep_initial = int(pool_kernel), int(keep_recent), int(keep_initial)
         self.pooled = None
         self.scores = torch.empty((Lyr, p.n_q_heads, T), dtype=torch.float32, device=dev)
         self.lse = torch.empty((Lyr, p.n_q_heads, T), dtype=torch.float32, device=dev)
@@ -306,12 +308,13 @@ class CompressionPass:
             kvcrush_select_pages(self.problem, self._selection_scores(scores), self.sigs, self.page_size,
                                  self.budget_imp, self.budget_rep, self.cu_kept, self.idx, kind=self.kind,
                                  anchor_mode=self.anchor_mode, anchor_bits=self.anchor_bits,
+                                 keep_initial=self.keep_initial, keep_recent=self.keep_recent,
                                  workspace=self.workspace, status=self.status)
             return
         kvcrush_select(self.problem, self._selection_scores(scores), self.sigs, self.budget_imp,
                        self.budget_rep, self.cu_kept, self.idx, kind=self.kind, anchor_mode=self.anchor_mode,
-                       anchor_bits=self.anchor_bits, keep_recent=self.keep_recent, workspace=self.workspace,
-                       status=self.status)
+                       anchor_bits=self.anchor_bits, keep_recent=self.keep_recent, keep_initial=self.keep_initial,
+                       workspace=self.workspace, status=self.status)
 
     def compact(self, k_cache, v_cache):
         if self.page_size:

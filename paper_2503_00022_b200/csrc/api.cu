@@ -129,7 +129,8 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
 
 int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
                    const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
-                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment, int keep_recent,
+                   int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                   int keep_initial, int keep_recent,
                    const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev,
                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
   Shape s;
@@ -141,12 +142,12 @@ int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, co
       anchor_mode != KVCRUSH_ANCHOR_EXPLICIT)
     return KVCRUSH_ERR_INVALID_ARG;
   if (anchor_mode == KVCRUSH_ANCHOR_EXPLICIT && !anchor_bits_dev) return KVCRUSH_ERR_INVALID_ARG;
-  if (keep_recent < 0) return KVCRUSH_ERR_INVALID_ARG;
+  if (keep_recent < 0 || keep_initial < 0) return KVCRUSH_ERR_INVALID_ARG;
   if (s.max_seqlen > 262144) return KVCRUSH_ERR_UNSUPPORTED;
   if (!workspace || workspace_bytes < select_workspace_bytes(s)) return KVCRUSH_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
   return launch_select(s, scores_dev, sigs_dev, budget_imp_dev, budget_rep_dev, anchor_mode, anchor_bits_dev,
-                       anchor_per_segment != 0, keep_recent, cu_kept_dev, idx_dev, kind_dev, workspace,
+                       anchor_per_segment != 0, keep_initial, keep_recent, cu_kept_dev, idx_dev, kind_dev, workspace,
                        static_cast<cudaStream_t>(stream));
 }
 
@@ -175,6 +176,7 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
 int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
                          int page_size, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
                          int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
+                         int keep_initial, int keep_recent,
                          const int32_t* cu_kept_dev, int32_t* page_idx_dev, uint8_t* kind_dev,
                          void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
   Shape s;
@@ -186,13 +188,14 @@ int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_d
       anchor_mode != KVCRUSH_ANCHOR_EXPLICIT)
     return KVCRUSH_ERR_INVALID_ARG;
   if (anchor_mode == KVCRUSH_ANCHOR_EXPLICIT && !anchor_bits_dev) return KVCRUSH_ERR_INVALID_ARG;
-  if (page_size < 1) return KVCRUSH_ERR_INVALID_ARG;
+  if (page_size < 1 || keep_initial < 0 || keep_recent < 0) return KVCRUSH_ERR_INVALID_ARG;
   if ((long long)page_size * s.W > kMaxPageWords) return KVCRUSH_ERR_UNSUPPORTED;
   if (((long long)s.max_seqlen + page_size - 1) / page_size > kMaxPagesPerSeq) return KVCRUSH_ERR_UNSUPPORTED;
   if (!workspace || workspace_bytes < select_workspace_bytes(s)) return KVCRUSH_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
   return launch_select_pages(s, scores_dev, sigs_dev, page_size, budget_imp_dev, budget_rep_dev, anchor_mode,
-                             anchor_bits_dev, anchor_per_segment != 0, cu_kept_dev, page_idx_dev, kind_dev,
+                             anchor_bits_dev, anchor_per_segment != 0, keep_initial, keep_recent, cu_kept_dev,
+                             page_idx_dev, kind_dev,
                              workspace, static_cast<cudaStream_t>(stream));
 }
 

@@ -66,19 +66,20 @@ int launch_signature(const Shape& s, const float* scores, const int32_t* sig_kee
 size_t select_workspace_bytes(const Shape& s);
 int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, const int32_t* budget_imp,
                   const int32_t* budget_rep, int anchor_mode, const uint32_t* anchor_bits, int anchor_per_segment,
-                  int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws, cudaStream_t stream);
+                  int keep_initial, int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws,
+                  cudaStream_t stream);
 
 // Order-preserving 64-bit keys of the token importance I(t), [n_layers][T] (first kernel of the selection stages).
-int launch_importance(const Shape& s, const float* scores, int keep_recent, unsigned long long* keys,
-                      cudaStream_t stream);
+int launch_importance(const Shape& s, const float* scores, int keep_initial, int keep_recent,
+                      unsigned long long* keys, cudaStream_t stream);
 
 // Page-granular selection and gather (a page = page_size consecutive tokens of one sequence).
 constexpr int kMaxPagesPerSeq = 8192;      // pages of one sequence the page kernel holds in shared memory
 constexpr int kMaxPageWords = 128;         // signature words of one page (page_size * W)
 int launch_select_pages(const Shape& s, const float* scores, const uint32_t* sigs, int page_size,
                         const int32_t* budget_imp, const int32_t* budget_rep, int anchor_mode,
-                        const uint32_t* anchor_bits, int anchor_per_segment, const int32_t* cu_kept,
-                        int32_t* page_idx, uint8_t* kind, void* ws, cudaStream_t stream);
+                        const uint32_t* anchor_bits, int anchor_per_segment, int keep_initial, int keep_recent,
+                        const int32_t* cu_kept, int32_t* page_idx, uint8_t* kind, void* ws, cudaStream_t stream);
 int launch_compact_pages(const Shape& s, const TensorView& K, const TensorView* V, int page_size,
                          const int32_t* cu_kept, const int32_t* page_idx, long long total_kept_pages,
                          const TensorView& K_out, const TensorView* V_out, cudaStream_t stream);

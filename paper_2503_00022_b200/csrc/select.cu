@@ -28,7 +28,8 @@ using sel::head_mask;
 constexpr int kMaxBins = 129;              // Hamming distances 0..128
 
 __global__ void __launch_bounds__(256)
-importance_kernel(Shape s, const float* __restrict__ scores, int keep_recent, unsigned long long* __restrict__ keys) {
+importance_kernel(Shape s, const float* __restrict__ scores, int keep_initial, int keep_recent,
+                  unsigned long long* __restrict__ keys) {
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= (long long)s.n_layers * s.T) return;
   const int layer = (int)(gid / s.T), tok = (int)(gid - (long long)layer * s.T);
@@ -50,9 +51,10 @@ importance_kernel(Shape s, const float* __restrict__ scores, int keep_recent, un
     }
   }
   total = __dadd_rn(total, 0.0);           // -0.0 -> +0.0
-  if (keep_recent > 0) {                   // the last keep_recent tokens of a sequence are important by decree
+  if (keep_recent > 0 || keep_initial > 0) {   // the first / last tokens of a sequence are important by decree
     const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
-    if (tok >= __ldg(s.cu_seqlens + seq + 1) - keep_recent) total = __longlong_as_double(0x7FF0000000000000LL);
+    if (tok >= __ldg(s.cu_seqlens + seq + 1) - keep_recent || tok < __ldg(s.cu_seqlens + seq) + keep_initial)
+      total = __longlong_as_double(0x7FF0000000000000LL);
   }
   const unsigned long long b = (unsigned long long)__double_as_longlong(total);
   keys[gid] = (b >> 63) ? ~b : (b | 0x8000000000000000ull);
@@ -305,10 +307,10 @@ select_segment_kernel(Shape s, SelectArgs a) {
 
 }  // namespace
 
-int launch_importance(const Shape& s, const float* scores, int keep_recent, unsigned long long* keys,
-                      cudaStream_t stream) {
+int launch_importance(const Shape& s, const float* scores, int keep_initial, int keep_recent,
+                      unsigned long long* keys, cudaStream_t stream) {
   const size_t n = (size_t)s.n_layers * s.T;
-  importance_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, scores, keep_recent, keys);
+  importance_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, scores, keep_initial, keep_recent, keys);
   return check_launch();
 }
 
@@ -319,12 +321,13 @@ size_t select_workspace_bytes(const Shape& s) {
 
 int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, const int32_t* budget_imp,
                   const int32_t* budget_rep, int anchor_mode, const uint32_t* anchor_bits, int anchor_per_segment,
-                  int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws, cudaStream_t stream) {
+                  int keep_initial, int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws,
+                  cudaStream_t stream) {
   if (s.T == 0) return KVCRUSH_OK;
   const size_t n = (size_t)s.n_layers * s.T;
   unsigned long long* keys = static_cast<unsigned long long*>(ws);
   int32_t* sorted = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(ws) + ((n * 8 + 255) / 256) * 256);
-  if (launch_importance(s, scores, keep_recent, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+  if (launch_importance(s, scores, keep_initial, keep_recent, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
 
   SelectArgs a{};
   a.keys = keys; a.sigs = sigs; a.budget_imp = budget_imp; a.budget_rep = budget_rep;

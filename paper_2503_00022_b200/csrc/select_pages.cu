@@ -40,6 +40,7 @@ struct PageArgs {
   int np_cap;                          // capacity of the per-page arrays (pages, multiple of 32)
   int sort_cap;                        // capacity of the sort array (power of two >= np_cap)
   int n_workers;                       // warps that own per-bit counters
+  int keep_initial, keep_recent;       // pages at both ends of a sequence that are important by decree
 };
 
 __device__ __forceinline__ double key_to_double(unsigned long long k) {
@@ -100,6 +101,7 @@ select_pages_kernel(Shape s, PageArgs a) {
       for (int j = 0; j < 8; ++j)
         if (i0 + j < n_tok) acc = __dadd_rn(acc, key_to_double(kk[j]));
     }
+    if (p < a.keep_initial || p >= n_pages - a.keep_recent) acc = __longlong_as_double(0x7FF0000000000000LL);
     pkeys[p] = double_to_key(acc);
   }
   for (int i = tid; i < n_words; i += kThreads) { imp_mask[i] = 0; rep_mask[i] = 0; }
@@ -235,17 +237,18 @@ select_pages_kernel(Shape s, PageArgs a) {
 
 int launch_select_pages(const Shape& s, const float* scores, const uint32_t* sigs, int page_size,
                         const int32_t* budget_imp, const int32_t* budget_rep, int anchor_mode,
-                        const uint32_t* anchor_bits, int anchor_per_segment, const int32_t* cu_kept,
-                        int32_t* page_idx, uint8_t* kind, void* ws, cudaStream_t stream) {
+                        const uint32_t* anchor_bits, int anchor_per_segment, int keep_initial, int keep_recent,
+                        const int32_t* cu_kept, int32_t* page_idx, uint8_t* kind, void* ws, cudaStream_t stream) {
   if (s.T == 0) return KVCRUSH_OK;
   unsigned long long* keys = static_cast<unsigned long long*>(ws);
-  if (launch_importance(s, scores, 0, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+  if (launch_importance(s, scores, 0, 0, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
 
   PageArgs a{};
   a.tok_keys = keys; a.sigs = sigs; a.budget_imp = budget_imp; a.budget_rep = budget_rep;
   a.anchor_mode = anchor_mode; a.anchor_bits = anchor_bits; a.anchor_per_segment = anchor_per_segment;
   a.cu_kept = cu_kept; a.page_idx = page_idx; a.kind = kind;
   a.P = page_size; a.PW = page_size * s.W;
+  a.keep_initial = keep_initial; a.keep_recent = keep_recent;
   const int max_pages = (s.max_seqlen + page_size - 1) / page_size;
   a.np_cap = ((max_pages + 31) / 32) * 32;
   a.sort_cap = 32;

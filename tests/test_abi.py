@@ -81,18 +81,21 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
     assert lib.kvcrush_signature(r(p), 0x100, None, None, 0x100, None, None, 0, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_signature(r(p), 0x100, 0x100, None, 0x100, None, None, 0, 0x100, None) == B.ERR_WORKSPACE
     # select: anchor mode range, explicit anchor needs bits, workspace
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 5, None, 0, 0, 0x100, 0x100, None, 0x100, 1 << 20,
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 5, None, 0, 0, 0, 0x100, 0x100, None, 0x100, 1 << 20,
                               0x100, None) == B.ERR_INVALID_ARG
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, B.ANCHOR_EXPLICIT, None, 0, 0, 0x100, 0x100, None,
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, B.ANCHOR_EXPLICIT, None, 0, 0, 0, 0x100, 0x100, None,
                               0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, 0, 0x100, 0x100, None, 0x100, 16,
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, 0, 0, 0x100, 0x100, None, 0x100, 16,
                               0x100, None) == B.ERR_WORKSPACE
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, -1, 0x100, 0x100, None, 0x100, 1 << 20,
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, 0, -1, 0x100, 0x100, None, 0x100, 1 << 20,
+                              0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, -1, 0, 0x100, 0x100, None, 0x100, 1 << 20,
                               0x100, None) == B.ERR_INVALID_ARG
     # page-granular select: page size, page vector too long, too many pages per sequence, workspace
-    sp = lambda ps, prob=p, ws=1 << 20: lib.kvcrush_select_pages(r(prob), 0x100, 0x100, ps, 0x100, 0x100, 0, None, 0, 0x100,
-                                                                 0x100, None, 0x100, ws, 0x100, None)
+    sp = lambda ps, prob=p, ws=1 << 20, ki=0: lib.kvcrush_select_pages(r(prob), 0x100, 0x100, ps, 0x100, 0x100, 0, None, 0,
+                                                                       ki, 0, 0x100, 0x100, None, 0x100, ws, 0x100, None)
     assert sp(0) == B.ERR_INVALID_ARG
+    assert sp(8, ki=-1) == B.ERR_INVALID_ARG
     assert sp(256) == B.ERR_UNSUPPORTED
     assert sp(8, ws=16) == B.ERR_WORKSPACE
     long_seq = _problem(cu=[0, 100000])

@@ -34,6 +34,7 @@ def test_random_selection_problems_are_bit_exact(B):
         ties = int(g.choice([0, 0, 2, 5]))
         mode = int(g.integers(0, 3))
         keep_recent = int(g.choice([0, 0, 3, 40]))
+        keep_initial = int(g.choice([0, 0, 4, 33]))
         b_imp = np.asarray([int(g.integers(0, L + 1)) for L in seqlens], dtype=np.int32)
         b_rep = np.asarray([int(g.integers(0, max(1, L - bi + 1))) for L, bi in zip(seqlens, b_imp)], dtype=np.int32)
         if case % 7 == 0:
@@ -47,7 +48,8 @@ def test_random_selection_problems_are_bit_exact(B):
         explicit = inputs.random_anchor_bits(Hq, 500 + case)
         prob = B.Problem(n_layers, Hq, Hkv, 16, seqlens, device=dev)
         cp = B.CompressionPass(prob, b_imp[None], b_rep[None], anchor_mode=mode,
-                               anchor_bits=explicit if mode == B.ANCHOR_EXPLICIT else None, keep_recent=keep_recent)
+                               anchor_bits=explicit if mode == B.ANCHOR_EXPLICIT else None, keep_recent=keep_recent,
+                               keep_initial=keep_initial)
         ds = torch.from_numpy(scores).to(dev)
         cp.signature(ds)
         cp.select(ds)
@@ -58,9 +60,10 @@ def test_random_selection_problems_are_bit_exact(B):
             for s, L in enumerate(seqlens):
                 s32 = np.ascontiguousarray(scores[l][:, cu[s]:cu[s + 1]])
                 sig = O.signatures(s32, O.thresholds(s32, int(b_imp[s] + b_rep[s])))
-                ctx = (case, Hq, Hkv, seqlens, b_imp.tolist(), b_rep.tolist(), ties, mode, keep_recent, l, s)
+                ctx = (case, Hq, Hkv, seqlens, b_imp.tolist(), b_rep.tolist(), ties, mode, keep_recent, keep_initial, l, s)
                 assert np.array_equal(sigs[l, cu[s]:cu[s + 1]], sig), ctx
-                idx, kind = O.select(s32, sig, int(b_imp[s]), int(b_rep[s]), Hkv, mode, explicit, keep_recent=keep_recent)
+                idx, kind = O.select(s32, sig, int(b_imp[s]), int(b_rep[s]), Hkv, mode, explicit, keep_recent=keep_recent,
+                                     keep_initial=keep_initial)
                 assert np.array_equal(cp.kept(l, s), idx.astype(np.int32)), ctx
                 seg = l * n_seqs + s
                 lo, hi = int(cp.cu_kept_host[seg]), int(cp.cu_kept_host[seg + 1])

@@ -18,13 +18,14 @@ def B():
     return binding
 
 
-def _run_pages(B, scores, Hkv, seqlens, P, b_imp, b_rep, mode=0, explicit=None):
+def _run_pages(B, scores, Hkv, seqlens, P, b_imp, b_rep, mode=0, explicit=None, keep=(0, 0)):
     import torch
     dev = torch.device("cuda:0")
     n_layers, Hq, _ = scores.shape
     prob = B.Problem(n_layers, Hq, Hkv, 16, seqlens, device=dev)
     cp = B.CompressionPass(prob, b_imp, b_rep, anchor_mode=mode,
-                           anchor_bits=explicit if mode == B.ANCHOR_EXPLICIT else None, page_size=P)
+                           anchor_bits=explicit if mode == B.ANCHOR_EXPLICIT else None, page_size=P,
+                           keep_initial=keep[0], keep_recent=keep[1])
     ds = torch.from_numpy(scores).to(dev)
     cp.signature(ds)
     cp.select(ds)
@@ -33,7 +34,7 @@ def _run_pages(B, scores, Hkv, seqlens, P, b_imp, b_rep, mode=0, explicit=None):
     return cp
 
 
-def _check_pages(cp, scores, Hkv, seqlens, P, b_imp, b_rep, mode=0, explicit=None, ctx=None):
+def _check_pages(cp, scores, Hkv, seqlens, P, b_imp, b_rep, mode=0, explicit=None, ctx=None, keep=(0, 0)):
     n_layers = scores.shape[0]
     cu = np.concatenate([[0], np.cumsum(seqlens)])
     b_imp = np.broadcast_to(np.asarray(b_imp), (n_layers, len(seqlens)))
@@ -43,7 +44,7 @@ def _check_pages(cp, scores, Hkv, seqlens, P, b_imp, b_rep, mode=0, explicit=Non
             s32 = np.ascontiguousarray(scores[l][:, cu[s]:cu[s + 1]])
             bi, br = int(b_imp[l, s]), int(b_rep[l, s])
             sig = O.signatures(s32, O.thresholds(s32, (bi + br) * P))
-            idx, kind = O.select_pages(s32, sig, P, bi, br, Hkv, mode, explicit)
+            idx, kind = O.select_pages(s32, sig, P, bi, br, Hkv, mode, explicit, keep_initial=keep[0], keep_recent=keep[1])
             np.testing.assert_array_equal(cp.kept(l, s), idx.astype(np.int32), err_msg=str((ctx, l, s)))
             seg = l * len(seqlens) + s
             lo, hi = int(cp.cu_kept_host[seg]), int(cp.cu_kept_host[seg + 1])
@@ -111,9 +112,22 @@ def test_random_page_problems_are_bit_exact(B):
             b_rep[:] = 1                                   # one bucket holding every grouped page
         scores = _scores(1, Hq, seqlens, 5000 + 20 * case, ties=ties)
         explicit = inputs.random_anchor_bits(Hq, 600 + case)
-        cp = _run_pages(B, scores, Hkv, seqlens, P, b_imp[None], b_rep[None], mode, explicit)
+        keep = (int(g.choice([0, 0, 1, 3])), int(g.choice([0, 0, 2, 5])))
+        cp = _run_pages(B, scores, Hkv, seqlens, P, b_imp[None], b_rep[None], mode, explicit, keep)
         _check_pages(cp, scores, Hkv, seqlens, P, b_imp[None], b_rep[None], mode, explicit,
-                     ctx=(case, Hq, Hkv, P, seqlens, b_imp.tolist(), b_rep.tolist(), mode, ties))
+                     ctx=(case, Hq, Hkv, P, seqlens, b_imp.tolist(), b_rep.tolist(), mode, ties, keep), keep=keep)
+
+
+def test_paged_budget_of_table1(B):
+    # 672 tokens = 32 initial + 512 middle + 128 recent at page size 32: 1 + 16 + 4 pages, 4 of the middle by KVCrush
+    seqlens = [4000, 2500]
+    scores = _scores(2, 32, seqlens, 88)
+    b_imp, b_rep = np.asarray([[17, 17]], dtype=np.int32), np.asarray([[4, 4]], dtype=np.int32)
+    cp = _run_pages(B, scores, 8, seqlens, 32, b_imp, b_rep, keep=(1, 4))
+    _check_pages(cp, scores, 8, seqlens, 32, b_imp, b_rep, keep=(1, 4))
+    for s, L in enumerate(seqlens):
+        n_pages = (L + 31) // 32
+        assert {0} | set(range(n_pages - 4, n_pages)) <= set(cp.kept(0, s).tolist())
 
 
 def test_widest_page_vector_and_most_pages(B):
