@@ -282,8 +282,12 @@ def run_ours(args, w):
         pages = np.maximum((b_imp + b_rep) // args.page_size, 1)
         b_rep = (pages // 2).astype(np.int32)
         b_imp = (pages - b_rep).astype(np.int32)
+    unit = max(args.page_size, 1)                         # decree lengths are given in tokens; pages in page mode
+    keep_recent = max(args.window, args.keep_recent) // unit
+    keep_initial = args.keep_initial // unit
     cp = B.CompressionPass(prob, b_imp[None, :], b_rep[None, :], cache_dtype=tc, impl=B.SCORE_AUTO,
-                           pool_kernel=args.pool, keep_recent=args.window, page_size=args.page_size)
+                           pool_kernel=args.pool, keep_recent=keep_recent, page_size=args.page_size,
+                           keep_initial=keep_initial)
     torch.cuda.synchronize()
 
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
@@ -359,7 +363,8 @@ def run_ours(args, w):
         pr = B.Problem(nl, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seqlens, causal=w.causal, device=dev,
                        query_window=args.window)
         passes.append(B.CompressionPass(pr, b_imp[None, :], b_rep[None, :], cache_dtype=tc, impl=B.SCORE_AUTO,
-                                        pool_kernel=args.pool, keep_recent=args.window, page_size=args.page_size))
+                                        pool_kernel=args.pool, keep_recent=keep_recent, page_size=args.page_size,
+                                        keep_initial=keep_initial))
     equal_chunks = all(bounds[c + 1] - bounds[c] == bounds[1] - bounds[0] for c in range(n_chunks))
     h_idx = [torch.empty(passes[0].idx.shape, dtype=torch.int32, pin_memory=True) for _ in range(n_chunks)]
     h_ko = [torch.empty(passes[0].k_out.shape, dtype=tc, pin_memory=True) for _ in range(n_chunks)]
@@ -465,7 +470,8 @@ def run_ours(args, w):
                    "budget_per_seq": [int(b_imp[0] + b_rep[0])], "cache_dtype": w.cache_dtype,
                    "l2": "inputs larger than L2 (%.1f GiB resident per step)" % (h2d / 2 ** 30),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "query_window": args.window, "pool_kernel": args.pool, "page_size": args.page_size},
+                   "query_window": args.window, "pool_kernel": args.pool, "page_size": args.page_size,
+                   "keep_initial": args.keep_initial, "keep_recent": max(args.window, args.keep_recent)},
         "layer_tokens_per_s": tokens * w.n_layers / (ms_per_step * 1e-3),
         "roofline": roofline, "stages": stages, "cpu_baseline": cpu,
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -495,6 +501,8 @@ def main():
     ap.add_argument("--pool", type=int, default=0, help="max-pool the per-head scores with this odd kernel width (0 = off)")
     ap.add_argument("--page-size", type=int, default=0,
                     help="evict whole pages of this many tokens (8 = the paper's chunks, 32 = its pages; 0 = token level)")
+    ap.add_argument("--keep-initial", type=int, default=0, help="first tokens of every sequence kept by decree (attention sinks)")
+    ap.add_argument("--keep-recent", type=int, default=0, help="last tokens of every sequence kept by decree")
     args = ap.parse_args()
     if args.page_size and args.window:
         ap.error("--page-size and --window are separate modes")
