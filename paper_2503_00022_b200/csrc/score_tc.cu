@@ -21,8 +21,8 @@
 //   * TMEM holds four 128-column accumulators, two per half, so the tensor core fills one buffer of a half
 //     while an epilogue group drains the other.
 //
-// Roles: warp 0 fetches + decodes items and issues TMA loads; warp 1 (one lane) issues tcgen05.mma;
-// warps 2..17 are four epilogue groups (half x buffer parity) of 128 threads, thread = TMEM lane = one
+// Roles: warp 0 fetches + decodes items and issues TMA loads; warps 1 and 2 (one lane each) issue the
+// tcgen05.mma of stationary half 0 and 1; warps 3..18 are four epilogue groups (half x buffer parity) of 128 threads, thread = TMEM lane = one
 // query row (sweep 1) or one key column (sweep 2).  All synchronisation is by mbarriers with bounded
 // waits: a role that gives up sets the CTA's abort flag, every other wait then ends, the CTA reports
 // through the status word, drains its copies, frees TMEM and returns.
@@ -40,7 +40,8 @@ using namespace tc;
 constexpr int kTile = 128;
 constexpr int kBlockRows = 2 * kTile;        // stationary rows per work item
 constexpr int kEpiWarps = 16;
-constexpr int kThreads = 64 + kEpiWarps * 32;
+constexpr int kIssueWarps = 2;                // one tcgen05.mma issuer per stationary half
+constexpr int kThreads = 32 * (1 + kIssueWarps) + kEpiWarps * 32;
 constexpr int kRing = 4;                     // streamed tiles in flight
 constexpr uint32_t kTmemCols = 512;          // 4 accumulators x 128 fp32 columns
 
@@ -78,7 +79,7 @@ struct PAux {
   unsigned long long item_full[2], item_empty[2];
   unsigned long long pair_bar[2];                     // both groups of one half (8 warps)
   unsigned long long group_bar[4];                    // one group (4 warps)
-  unsigned long long drain;
+  unsigned long long drain[kIssueWarps];
   uint32_t tmem_base;
   int abort_flag;
   int item[2][8];                                     // layer, head, seq, block, n_tiles (layer < 0: no more work)
@@ -137,10 +138,10 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (lane == 0) {
       // a launch that already failed somewhere is not worth finishing
       aux->abort_flag = *reinterpret_cast<volatile int32_t*>(a.status) != 0;
-      for (int i = 0; i < kRing; ++i) { mbar_init(smem_u32(&aux->full[i]), 1); mbar_init(smem_u32(&aux->empty[i]), 1); }
+      for (int i = 0; i < kRing; ++i) { mbar_init(smem_u32(&aux->full[i]), 1); mbar_init(smem_u32(&aux->empty[i]), kIssueWarps); }
       mbar_init(smem_u32(&aux->fixed_full), 1);
-      mbar_init(smem_u32(&aux->fixed_empty), 1);
-      mbar_init(smem_u32(&aux->drain), 1);
+      mbar_init(smem_u32(&aux->fixed_empty), kIssueWarps);
+      for (int i = 0; i < kIssueWarps; ++i) mbar_init(smem_u32(&aux->drain[i]), 1);
       for (int i = 0; i < 4; ++i) {
         mbar_init(smem_u32(&aux->acc_full[i]), 1);
         mbar_init(smem_u32(&aux->acc_empty[i]), 4);
@@ -148,7 +149,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       for (int i = 0; i < 2; ++i) {
         mbar_init(smem_u32(&aux->item_full[i]), 1);
-        mbar_init(smem_u32(&aux->item_empty[i]), 1 + kEpiWarps);
+        mbar_init(smem_u32(&aux->item_empty[i]), kIssueWarps + kEpiWarps);
         mbar_init(smem_u32(&aux->pair_bar[i]), 8);
       }
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -233,11 +234,15 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (issued_item > 0)
         for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->fixed_full), (issued_item - 1) & 1); ++i) {}
     }
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
+  } else if (warp <= kIssueWarps) {
+    // ------------------------------ MMA issuers ------------------------------
+    // One thread per stationary half.  tcgen05.mma blocks its issuer while the tensor core's queue is full, and
+    // the queue is short, so a lone issuer leaves the pipe idle whenever it has to poll a barrier; with two
+    // issuers one polls while the other's instructions are queued.
     if (lane == 0) {
+      const int hf = warp - 1;
       constexpr uint32_t idesc = make_idesc(kTile, kTile);
-      int n_item = 0, n_stream = 0, cnt[2] = {0, 0};
+      int n_item = 0, n_stream = 0, cnt = 0;
       bool ok = true;
       while (ok) {
         const int slot = n_item & 1;
@@ -252,10 +257,12 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         ok = mbar_wait(smem_u32(&aux->fixed_full), n_item & 1, abort_flag);
         for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
           const int rs = n_stream % kRing;
+          // also when this half skips the tile: the wait keeps the issuer from running a whole ring ahead of
+          // the other one, whose arrival on empty[rs] must fall into the same phase as this one's
           ok = mbar_wait(smem_u32(&aux->full[rs]), (n_stream / kRing) & 1, abort_flag);
-          for (int hf = 0; ok && hf < 2; ++hf) {
-            if (!g.active(hf, i)) continue;
-            const int c = cnt[hf]++;
+          if (!ok) break;
+          if (g.active(hf, i)) {
+            const int c = cnt++;
             const int buf = 2 * hf + (c & 1);
             ok = mbar_wait(smem_u32(&aux->acc_empty[buf]), ((c >> 1) & 1) ^ 1, abort_flag);
             if (!ok) break;
@@ -269,7 +276,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             }
             umma_commit(smem_u32(&aux->acc_full[buf]));
           }
-          if (!ok) break;
+          // this issuer is done with the ring slot (a commit with nothing pending arrives at once)
           umma_commit(smem_u32(&aux->empty[rs]));
         }
         if (!ok) break;
@@ -278,13 +285,13 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       if (*abort_flag) {
         // wait (bounded) until every MMA already issued has retired before TMEM and shared memory go away
-        umma_commit(smem_u32(&aux->drain));
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->drain), 0); ++i) {}
+        umma_commit(smem_u32(&aux->drain[hf]));
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->drain[hf]), 0); ++i) {}
       }
     }
   } else {
     // ------------------------------ epilogue groups ------------------------------
-    const int gi = (warp - 2) >> 2;                // group = half * 2 + parity
+    const int gi = (warp - 1 - kIssueWarps) >> 2;  // group = half * 2 + parity
     const int hf = gi >> 1, par = gi & 1;
     const int quarter = warp & 3;                  // TMEM lanes this warp may read
     const int r = quarter * 32 + lane;             // row of the accumulator = TMEM lane = index inside the group
