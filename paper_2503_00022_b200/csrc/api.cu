@@ -85,7 +85,6 @@ int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, c
   if ((rc = make_view(K, s.D, &k)) != KVCRUSH_OK) return rc;
   if (!scores_dev || !status_dev) return KVCRUSH_ERR_INVALID_ARG;
   if (q.dtype != k.dtype) return KVCRUSH_ERR_INVALID_ARG;
-  if (q.dtype != KVCRUSH_BF16 && q.dtype != KVCRUSH_FP32) return KVCRUSH_ERR_UNSUPPORTED;
   if (impl != KVCRUSH_SCORE_AUTO && impl != KVCRUSH_SCORE_SIMT && impl != KVCRUSH_SCORE_TENSOR)
     return KVCRUSH_ERR_INVALID_ARG;
   if (!workspace || workspace_bytes < score_ws(s)) return KVCRUSH_ERR_WORKSPACE;

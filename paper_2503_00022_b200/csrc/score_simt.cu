@@ -1,6 +1,6 @@
 // Stage 1 on CUDA cores (fp32 arithmetic): attention column sums (Algorithm 1 of the paper,
 // "attention weights" and "normalized attention score" steps).  Serves fp32 inputs and shapes the
-// tensor-core kernels do not cover; the S x S matrix is never stored.
+// tensor-core kernels do not cover (bf16 and fp16 inputs are widened on load); the S x S matrix is never stored.
 //
 //   lse_rows_kernel   one warp per query row j: lanes take keys t, t+32, ..; each lane keeps an
 //                     online (max, sum) pair in the log2 domain; lse2(j) = log2 sum_t 2^(s2(j,t))
@@ -8,6 +8,7 @@
 //   colsum_kernel     one warp per key t: lanes take queries j, j+32, ..; accumulates
 //                     2^(s2(j,t) - lse2(j)) = A(j,t) and reduces over the warp.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 
@@ -36,6 +37,18 @@ __device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16* p, flo
   for (int i = 0; i < 4; ++i) {
     v[2 * i] = __uint_as_float(w[i] << 16);
     v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+template <>
+__device__ __forceinline__ void load8<__half>(const __half* p, float (&v)[8]) {
+  const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+    v[2 * i] = f.x;
+    v[2 * i + 1] = f.y;
   }
 }
 
@@ -162,6 +175,8 @@ int launch_score_simt(const Shape& s, const TensorView& Q, const TensorView& K, 
     return run<float>(s, Q, K, scale_log2, lse_in, lse_in_mul, lse2_ws, scores, lse_out, normalize, stream);
   if (Q.dtype == KVCRUSH_BF16)
     return run<__nv_bfloat16>(s, Q, K, scale_log2, lse_in, lse_in_mul, lse2_ws, scores, lse_out, normalize, stream);
+  if (Q.dtype == KVCRUSH_FP16)
+    return run<__half>(s, Q, K, scale_log2, lse_in, lse_in_mul, lse2_ws, scores, lse_out, normalize, stream);
   return KVCRUSH_ERR_UNSUPPORTED;
 }
 

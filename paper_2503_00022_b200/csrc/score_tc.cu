@@ -1,4 +1,4 @@
-// Stage 1 on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16 Q/K, head_dim 64 or 128.
+// Stage 1 on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16 or fp16 Q/K, head_dim 64 or 128.
 //
 // Attention column sums (Algorithm 1 of the paper: A_h = softmax(Q_h K_h^T / sqrt(d_k)), then the per-token
 // sum of A_h over the queries) without ever storing the S x S matrix: two sweeps that both recompute
@@ -54,6 +54,7 @@ struct PersistArgs {
   float* lse_nat_out;      // sweep 1: optional natural-log copy
   float* scores;           // sweep 2 output
   int normalize;
+  int bf16;                // operand type of Q and K: bf16 (1) or fp16 (0)
   int max_blocks;          // ceil(max_seqlen / 256)
   int n_items;             // (sequence, 256-row block) pairs of one (layer, head)
   int total_items;         // n_items * n_layers * Hq
@@ -241,7 +242,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // issuers one polls while the other's instructions are queued.
     if (lane == 0) {
       const int hf = warp - 1;
-      constexpr uint32_t idesc = make_idesc(kTile, kTile);
+      const uint32_t idesc = make_idesc(kTile, kTile, a.bf16 != 0);
       int n_item = 0, n_stream = 0, cnt = 0;
       bool ok = true;
       while (ok) {
@@ -444,7 +445,7 @@ int launch_persist(const CUtensorMap& mq, const CUtensorMap& mk, const PersistAr
 size_t score_tensor_counter_bytes() { return 256; }
 
 bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorView& K) {
-  if (Q.dtype != KVCRUSH_BF16 || K.dtype != KVCRUSH_BF16) return false;
+  if (Q.dtype != K.dtype || (Q.dtype != KVCRUSH_BF16 && Q.dtype != KVCRUSH_FP16)) return false;
   if (s.D != 64 && s.D != 128) return false;
   if (s.T < 1) return false;
   return encode_fn() != nullptr;
@@ -465,7 +466,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
       cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sms < 1)
     return KVCRUSH_ERR_CUDA;
   PersistArgs a{};
-  a.s = s; a.scale_log2 = scale_log2; a.normalize = normalize; a.status = status; a.scores = scores;
+  a.s = s; a.scale_log2 = scale_log2; a.normalize = normalize; a.bf16 = Q.dtype == KVCRUSH_BF16; a.status = status; a.scores = scores;
   a.max_blocks = (s.max_seqlen + kBlockRows - 1) / kBlockRows;
   // work items per (layer, head): every 256-row block for the column sweep; for the row sweep only the
   // blocks that hold voting queries

@@ -283,9 +283,11 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
   return d;
 }
 
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, M x N.
-__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+// kind::f16 instruction descriptor: fp32 accumulate, both operands K-major and of one type (bf16 x bf16 or
+// fp16 x fp16: format code 1 or 0 in the A and B fields), M x N.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool bf16) {
+  return (1u << 4) | ((bf16 ? 1u : 0u) << 7) | ((bf16 ? 1u : 0u) << 10) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(m >> 4) << 24);
 }
 
 
@@ -350,7 +352,7 @@ inline EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 4-D view (channel, token, head, layer) of a token-major bf16 tensor; box = 64 channels x 128 tokens.
+// 4-D view (channel, token, head, layer) of a token-major bf16 or fp16 tensor; box = 64 channels x 128 tokens.
 inline bool make_map(CUtensorMap* map, const TensorView& t, int D, int T, int H, int n_layers) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
@@ -359,7 +361,7 @@ inline bool make_map(CUtensorMap* map, const TensorView& t, int D, int T, int H,
   const cuuint64_t gstride[3] = {stride_bytes(t.st), stride_bytes(t.sh), stride_bytes(t.sl)};
   const cuuint32_t box[4] = {64, 128u, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(t.ptr), gdim, gstride, box, estr,
+  return enc(map, t.dtype == KVCRUSH_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(t.ptr), gdim, gstride, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -73,7 +73,9 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
     # score: NULL outputs, misaligned tensor, dtype mismatch / unsupported, missing workspace
     assert lib.kvcrush_score(r(p), r(t), r(t), None, None, None, 0, 0, None, 0, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_score(r(p), r(odd), r(t), None, 0x100, None, 0, 0, 0x100, 1 << 20, 0x100, None) == B.ERR_MISALIGNED
-    assert lib.kvcrush_score(r(p), r(f16), r(f16), None, 0x100, None, 0, 0, 0x100, 1 << 20, 0x100, None) == B.ERR_UNSUPPORTED
+    f32 = B.TensorStruct(0x10000, B.FP32, 0, 100 * 8 * 64, 8 * 64, 64)
+    assert lib.kvcrush_score(r(p), r(f32), r(f32), None, 0x100, None, 0, B.SCORE_TENSOR, 0x100, 1 << 20, 0x100,
+                             None) == B.ERR_UNSUPPORTED          # the tensor-core kernels take bf16 / fp16 only
     assert lib.kvcrush_score(r(p), r(t), r(f16), None, 0x100, None, 0, 0, 0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_score(r(p), r(t), r(t), None, 0x100, None, 0, 0, None, 0, 0x100, None) == B.ERR_WORKSPACE
     assert lib.kvcrush_score(r(p), r(t), r(t), None, 0x100, None, 0, 7, 0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG

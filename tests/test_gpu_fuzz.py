@@ -83,7 +83,8 @@ def test_random_score_problems_match_oracle_and_cuda_core_path(B):
         causal = bool(g.integers(0, 4) > 0)
         window = int(g.choice([0, 0, 17, 130]))
         n_layers = int(g.integers(1, 3))
-        w = inputs.Workload(f"fz{case}", n_layers, Hq, Hkv, D, seqlens, inputs.BF16, inputs.BF16, 0.25,
+        qk = inputs.FP16 if case % 3 == 2 else inputs.BF16
+        w = inputs.Workload(f"fz{case}", n_layers, Hq, Hkv, D, seqlens, qk, inputs.BF16, 0.25,
                             base_seed=7000 + case, causal=causal)
         lis, q, k, _, _ = TL.stack_layers(w, range(n_layers), with_cache=False)
         prob = B.Problem(n_layers, Hq, Hkv, D, seqlens, causal=causal, device=dev, query_window=window)
@@ -97,7 +98,7 @@ def test_random_score_problems_match_oracle_and_cuda_core_path(B):
             torch.cuda.synchronize()
             assert status.cpu().tolist()[0] == 0
             out[name] = sc.cpu().numpy()
-        ctx = (case, D, Hq, Hkv, seqlens, causal, window)
+        ctx = (case, D, Hq, Hkv, seqlens, causal, window, qk)
         np.testing.assert_allclose(out["tensor"], out["simt"], rtol=3e-4, atol=2e-6, err_msg=str(ctx))
         cu = w.cu_seqlens
         for l, li in enumerate(lis):
