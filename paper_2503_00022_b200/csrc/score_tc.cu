@@ -113,6 +113,7 @@ struct Geo {
   // does streamed tile `it` contribute to half `hf` (causal: the half's own tile index is 2*blk + hf)
   __device__ __forceinline__ bool active(int hf, int it) const {
     if (hf == 1 && !half1) return false;
+    if (!kColsum && blk * kBlockRows + hf * kTile + kTile <= ws) return false;   // no query of this half votes
     if (!causal) return true;
     return kColsum ? first_stream + it >= 2 * blk + hf : it <= 2 * blk + hf;
   }
