@@ -121,7 +121,8 @@ int kvcrush_workspace_size(const kvcrush_problem_t* problem, int stage, size_t* 
  * The S x S matrix is never stored: a first sweep computes the log-sum-exp of every
  * query row, a second sweep recomputes the logits and accumulates exp(s - lse).
  *   Q, K        token-major tensors with n_q_heads / n_kv_heads heads, same dtype
- *               (BF16, FP16 or FP32).  Tensor-core kernels: BF16 or FP16, head_dim 64 or 128.
+ *               (BF16, FP16 or FP32).  Tensor-core kernels: BF16 or FP16, head_dim a
+ *               multiple of 8 up to 128 (full speed at 64 and 128).
  *   lse_in_dev  optional [n_layers][n_q_heads][T] float32 natural-log row
  *               log-sum-exp of the scaled logits (as a prefill attention kernel
  *               returns it); when given the first sweep is skipped.

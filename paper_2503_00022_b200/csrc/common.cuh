@@ -48,7 +48,7 @@ __device__ __forceinline__ int seq_of_token(const int32_t* __restrict__ cu, int 
 
 // ---- stage launchers (defined in the per-stage .cu files) -------------------------------------------
 
-// score: SIMT fp32 kernels (any dtype/shape) and tcgen05 kernels (bf16, D in {64,128}).
+// score: SIMT fp32 kernels (any dtype/shape) and tcgen05 kernels (bf16 or fp16, D a multiple of 8 up to 128).
 // lse2_ws: [n_layers][Hq][T] float32 row log-sum-exp in the log2 domain (written unless lse_in is given).
 int launch_score_simt(const Shape& s, const TensorView& Q, const TensorView& K, float scale_log2,
                       const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores, float* lse_out,

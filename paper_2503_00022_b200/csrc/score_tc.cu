@@ -1,4 +1,6 @@
-// Stage 1 on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16 or fp16 Q/K, head_dim 64 or 128.
+// Stage 1 on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16 or fp16 Q/K, head_dim up to 128
+// (a multiple of 8; widths other than 64 and 128 run in the next larger kernel: the TMA boxes read zeros past
+// the last channel, and zeros add nothing to a dot product).
 //
 // Attention column sums (Algorithm 1 of the paper: A_h = softmax(Q_h K_h^T / sqrt(d_k)), then the per-token
 // sum of A_h over the queries) without ever storing the S x S matrix: two sweeps that both recompute
@@ -447,7 +449,7 @@ size_t score_tensor_counter_bytes() { return 256; }
 
 bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorView& K) {
   if (Q.dtype != K.dtype || (Q.dtype != KVCRUSH_BF16 && Q.dtype != KVCRUSH_FP16)) return false;
-  if (s.D != 64 && s.D != 128) return false;
+  if (s.D < 8 || s.D > 128 || s.D % 8 != 0) return false;      // other widths ride in the 64- or 128-wide kernel
   if (s.T < 1) return false;
   return encode_fn() != nullptr;
 }
@@ -486,7 +488,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
   if (!lse_in) {
     a.lse2_out = lse2_ws; a.lse_nat_out = lse_out; a.counter = counters;
     a.n_items = (int)items_row; a.total_items = (int)(items_row * s.n_layers * s.Hq);
-    rc = s.D == 128 ? launch_persist<128, false>(mq, mk, a, n_sms, stream) : launch_persist<64, false>(mq, mk, a, n_sms, stream);
+    rc = s.D > 64 ? launch_persist<128, false>(mq, mk, a, n_sms, stream) : launch_persist<64, false>(mq, mk, a, n_sms, stream);
     if (rc != KVCRUSH_OK) return rc;
     a.lse = lse2_ws; a.lse_mul = 1.f;
   } else {
@@ -494,7 +496,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
   }
   a.counter = counters + 1;
   a.n_items = (int)items_col; a.total_items = (int)(items_col * s.n_layers * s.Hq);
-  return s.D == 128 ? launch_persist<128, true>(mq, mk, a, n_sms, stream) : launch_persist<64, true>(mq, mk, a, n_sms, stream);
+  return s.D > 64 ? launch_persist<128, true>(mq, mk, a, n_sms, stream) : launch_persist<64, true>(mq, mk, a, n_sms, stream);
 }
 
 }  // namespace kvc

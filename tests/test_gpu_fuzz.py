@@ -75,7 +75,7 @@ def test_random_score_problems_match_oracle_and_cuda_core_path(B):
     dev = torch.device("cuda:0")
     g = np.random.Generator(np.random.Philox(4048))
     for case in range(14):
-        D = int(g.choice([64, 128]))
+        D = int(g.choice([64, 128, 96, 80, 32, 128]))
         Hkv = int(g.choice([1, 2, 4]))
         Hq = Hkv * int(g.choice([1, 2, 4]))
         n_seqs = int(g.integers(1, 6))
@@ -133,3 +133,27 @@ def test_large_logits_stay_within_tolerance(B):
             c, _ = O.scores(inputs.widen(lis[0].q[a:b], w.qk_dtype), inputs.widen(lis[0].k[a:b], w.qk_dtype), True, scale=scale)
             ok = TL.within_score_tolerance(g[0][:, a:b], c)
             assert ok.all(), (impl, s_, np.argwhere(~ok)[:4], g[0][:, a:b][~ok][:4], c[~ok][:4])
+
+
+@pytest.mark.parametrize("D", [96, 80, 8])
+def test_head_dims_between_the_kernel_widths(B, D):
+    """head_dim 96 (Phi-3-mini, one of the paper's models) and other multiples of 8 run in the next wider tensor-core
+    kernel with the missing channels read as zeros."""
+    import torch
+    dev = torch.device("cuda:0")
+    w = inputs.Workload(f"d{D}", 1, 4, 2, D, (700, 129), inputs.BF16, inputs.BF16, 0.25, base_seed=300 + D)
+    lis, q, k, _, _ = TL.stack_layers(w, range(1), with_cache=False)
+    prob = B.Problem(1, 4, 2, D, w.seqlens, device=dev)
+    ws = torch.empty(B.kvcrush_workspace_size(prob, B.STAGE_SCORE), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    sc = torch.empty((1, 4, w.total_tokens), dtype=torch.float32, device=dev)
+    B.kvcrush_score(prob, TL.torch_storage(q, w.qk_dtype, dev), TL.torch_storage(k, w.qk_dtype, dev), sc,
+                    impl=B.SCORE_TENSOR, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0
+    got = sc.cpu().numpy()
+    cu = w.cu_seqlens
+    for s_, L in enumerate(w.seqlens):
+        a, b = int(cu[s_]), int(cu[s_ + 1])
+        c, _ = O.scores(inputs.widen(lis[0].q[a:b], w.qk_dtype), inputs.widen(lis[0].k[a:b], w.qk_dtype), True)
+        assert TL.within_score_tolerance(got[0][:, a:b], c).all(), (D, s_)
