@@ -333,6 +333,22 @@ class CompressionPass:
         if k_cache is not None:
             self.compact(k_cache, v_cache)
 
+    def capture(self, q, k, k_cache=None, v_cache=None, lse_in=None):
+        """Records one ``run`` into a CUDA graph: the library only enqueues kernels and one memset on the stream
+        it is given, so the whole pass replays as a single launch (worth it when the pass is short and launch
+        overhead shows).  The tensors must stay where they are; ``replay`` runs the pass on their current contents."""
+        import torch
+        self.run(q, k, k_cache, v_cache, lse_in)          # outside the capture: one-time kernel attribute calls
+        torch.cuda.synchronize()
+        self.check_status()
+        self._graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self._graph):
+            self.run(q, k, k_cache, v_cache, lse_in)
+        return self._graph
+
+    def replay(self):
+        self._graph.replay()
+
     def check_status(self):
         st = self.status.cpu().tolist()
         if st[0] != DEV_OK:
