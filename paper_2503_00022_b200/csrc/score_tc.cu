@@ -18,16 +18,18 @@
 //
 //   * one CTA per SM lives for the whole launch and pulls work items from an atomic counter, so TMEM
 //     allocation, barrier set-up and pipeline fill are paid once per SM instead of once per item;
-//   * an item is a 256-row block of the stationary operand (two 128-row halves).  Every streamed
-//     128-row tile is multiplied with both halves, which halves the L2 -> shared-memory traffic per logit;
-//   * TMEM holds four 128-column accumulators, two per half, so the tensor core fills one buffer of a half
-//     while an epilogue group drains the other.
+//   * an item is a 512-row block of the stationary operand (four 128-row quarters).  Every streamed
+//     128-row tile is multiplied with all four quarters, which quarters the L2 -> shared-memory traffic per
+//     logit compared with one tile pair per load;
+//   * TMEM holds one 128-column accumulator per quarter, owned by one epilogue group: a group needs no merge
+//     with another group, and while it waits for its accumulator to be refilled the other three keep the
+//     special-function unit busy.
 //
 // Roles: warp 0 fetches + decodes items and issues TMA loads; warps 1 and 2 (one lane each) issue the
-// tcgen05.mma of stationary half 0 and 1; warps 3..18 are four epilogue groups (half x buffer parity) of 128 threads, thread = TMEM lane = one
-// query row (sweep 1) or one key column (sweep 2).  All synchronisation is by mbarriers with bounded
-// waits: a role that gives up sets the CTA's abort flag, every other wait then ends, the CTA reports
-// through the status word, drains its copies, frees TMEM and returns.
+// tcgen05.mma of quarters 0-1 and 2-3; warps 3..18 are four epilogue groups (one per quarter) of 128 threads,
+// thread = TMEM lane = one query row (sweep 1) or one key column (sweep 2).  All synchronisation is by mbarriers
+// with bounded waits: a role that gives up sets the CTA's abort flag, every other wait then ends, the CTA
+// reports through the status word, drains its copies, frees TMEM and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -40,12 +42,13 @@ namespace {
 using namespace tc;
 
 constexpr int kTile = 128;
-constexpr int kBlockRows = 2 * kTile;        // stationary rows per work item
+constexpr int kQ = 4;                        // stationary 128-row quarters per work item
+constexpr int kBlockRows = kQ * kTile;       // stationary rows per work item
 constexpr int kEpiWarps = 16;
 constexpr int kIssueWarps = 2;                // one tcgen05.mma issuer per stationary half
 constexpr int kThreads = 32 * (1 + kIssueWarps) + kEpiWarps * 32;
-constexpr int kRing = 4;                     // streamed tiles in flight
-constexpr uint32_t kTmemCols = 512;          // 4 accumulators x 128 fp32 columns
+constexpr int kRing = 2;                     // streamed tiles in flight
+constexpr uint32_t kTmemCols = 512;          // one 128-column fp32 accumulator per quarter
 
 struct PersistArgs {
   Shape s;
@@ -57,8 +60,8 @@ struct PersistArgs {
   float* scores;           // sweep 2 output
   int normalize;
   int bf16;                // operand type of Q and K: bf16 (1) or fp16 (0)
-  int max_blocks;          // ceil(max_seqlen / 256)
-  int n_items;             // (sequence, 256-row block) pairs of one (layer, head)
+  int max_blocks;          // ceil(max_seqlen / kBlockRows)
+  int n_items;             // (sequence, stationary block) pairs of one (layer, head)
   int total_items;         // n_items * n_layers * Hq
   int* counter;            // work counter, zero at launch
   int32_t* status;
@@ -68,8 +71,8 @@ template <int D>
 struct PSmem {
   static constexpr int kTileBytes = kTile * D * 2;
   static constexpr int kBlockBytes = kTile * 128;
-  static constexpr int kFixedOff = 0;                            // two stationary halves
-  static constexpr int kRingOff = 2 * kTileBytes;
+  static constexpr int kFixedOff = 0;                            // the stationary quarters
+  static constexpr int kRingOff = kQ * kTileBytes;
   static constexpr int kAuxOff = kRingOff + kRing * kTileBytes;
   static constexpr int kAuxBytes = 10240;
   static constexpr int kTotal = kAuxOff + kAuxBytes + 1024;
@@ -78,16 +81,14 @@ struct PSmem {
 struct PAux {
   unsigned long long full[kRing], empty[kRing];
   unsigned long long fixed_full, fixed_empty;
-  unsigned long long acc_full[4], acc_empty[4];       // [half * 2 + parity]
+  unsigned long long acc_full[kQ], acc_empty[kQ];     // [quarter]
   unsigned long long item_full[2], item_empty[2];
-  unsigned long long pair_bar[2];                     // both groups of one half (8 warps)
-  unsigned long long group_bar[4];                    // one group (4 warps)
+  unsigned long long group_bar[kQ];                   // one epilogue group (4 warps)
   unsigned long long drain[kIssueWarps];
   uint32_t tmem_base;
   int abort_flag;
   int item[2][8];                                     // layer, head, seq, block, n_tiles (layer < 0: no more work)
-  alignas(16) float lse_sh[4][2][kTile];              // [group][buffer][query of the streamed tile]
-  alignas(16) float part[2][2][2][kTile];             // [half][item parity][value][row]
+  alignas(16) float lse_sh[kQ][2][kTile];             // [group][buffer][query of the streamed tile]
 };
 
 // Geometry of one work item, derived identically by every role.
@@ -95,32 +96,33 @@ template <bool kColsum>
 struct Geo {
   int layer, h, hk, t0, L, blk, first_stream, n_iter;
   int ws;                      // first query row that votes (0 without an observation window)
-  bool causal, half1;
+  bool causal;
+  int nq;                      // quarters of the block that hold rows of the sequence
   __device__ __forceinline__ Geo(const Shape& s, const int* it) {
     layer = it[0]; h = it[1]; hk = h / s.G; blk = it[3];
     const int seq = it[2], n_tiles = it[4];
     t0 = __ldg(s.cu_seqlens + seq);
     L = __ldg(s.cu_seqlens + seq + 1) - t0;
     causal = s.causal != 0;
-    half1 = blk * kBlockRows + kTile < L;                               // does the second half hold any row
+    nq = min(kQ, (L - blk * kBlockRows + kTile - 1) / kTile);
     ws = (s.window > 0 && L > s.window) ? L - s.window : 0;
     if (kColsum) {                                                      // stationary keys, streamed query tiles
-      first_stream = max(causal ? 2 * blk : 0, ws / kTile);
+      first_stream = max(causal ? kQ * blk : 0, ws / kTile);
       n_iter = n_tiles - first_stream;
     } else {                                                            // stationary queries, streamed key tiles
       first_stream = 0;
-      n_iter = causal ? min(2 * blk + 2, n_tiles) : n_tiles;
+      n_iter = causal ? min(kQ * blk + kQ, n_tiles) : n_tiles;
     }
   }
-  // does streamed tile `it` contribute to half `hf` (causal: the half's own tile index is 2*blk + hf)
-  __device__ __forceinline__ bool active(int hf, int it) const {
-    if (hf == 1 && !half1) return false;
-    if (!kColsum && blk * kBlockRows + hf * kTile + kTile <= ws) return false;   // no query of this half votes
+  // does streamed tile `it` contribute to quarter `qd` (causal: the quarter's own tile index is kQ*blk + qd)
+  __device__ __forceinline__ bool active(int qd, int it) const {
+    if (qd >= nq) return false;
+    if (!kColsum && blk * kBlockRows + qd * kTile + kTile <= ws) return false;   // no query of this quarter votes
     if (!causal) return true;
-    return kColsum ? first_stream + it >= 2 * blk + hf : it <= 2 * blk + hf;
+    return kColsum ? first_stream + it >= kQ * blk + qd : it <= kQ * blk + qd;
   }
-  __device__ __forceinline__ bool diag(int hf, int it) const {
-    return causal && (kColsum ? first_stream + it == 2 * blk + hf : it == 2 * blk + hf);
+  __device__ __forceinline__ bool diag(int qd, int it) const {
+    return causal && (kColsum ? first_stream + it == kQ * blk + qd : it == kQ * blk + qd);
   }
 };
 
@@ -146,7 +148,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       mbar_init(smem_u32(&aux->fixed_full), 1);
       mbar_init(smem_u32(&aux->fixed_empty), kIssueWarps);
       for (int i = 0; i < kIssueWarps; ++i) mbar_init(smem_u32(&aux->drain[i]), 1);
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < kQ; ++i) {
         mbar_init(smem_u32(&aux->acc_full[i]), 1);
         mbar_init(smem_u32(&aux->acc_empty[i]), 4);
         mbar_init(smem_u32(&aux->group_bar[i]), 4);
@@ -154,7 +156,6 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       for (int i = 0; i < 2; ++i) {
         mbar_init(smem_u32(&aux->item_full[i]), 1);
         mbar_init(smem_u32(&aux->item_empty[i]), kIssueWarps + kEpiWarps);
-        mbar_init(smem_u32(&aux->pair_bar[i]), 8);
       }
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -207,9 +208,8 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // the stationary buffer is free once every MMA of the previous item has retired
         ok = mbar_wait(smem_u32(&aux->fixed_empty), (n_item & 1) ^ 1, abort_flag);
         if (ok) {
-          const int n_half = g.half1 ? 2 : 1;
-          mbar_expect_tx(smem_u32(&aux->fixed_full), n_half * SL::kTileBytes);
-          for (int hf = 0; hf < n_half; ++hf)
+          mbar_expect_tx(smem_u32(&aux->fixed_full), g.nq * SL::kTileBytes);
+          for (int hf = 0; hf < g.nq; ++hf)
 #pragma unroll
             for (int kb = 0; kb < D / 64; ++kb)
               tma_load_4d(fixed_addr + hf * SL::kTileBytes + kb * SL::kBlockBytes, map_fixed, smem_u32(&aux->fixed_full),
@@ -240,13 +240,13 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
   } else if (warp <= kIssueWarps) {
     // ------------------------------ MMA issuers ------------------------------
-    // One thread per stationary half.  tcgen05.mma blocks its issuer while the tensor core's queue is full, and
-    // the queue is short, so a lone issuer leaves the pipe idle whenever it has to poll a barrier; with two
-    // issuers one polls while the other's instructions are queued.
+    // One thread per pair of stationary quarters.  tcgen05.mma blocks its issuer while the tensor core's queue is
+    // full, and the queue is short, so a lone issuer leaves the pipe idle whenever it has to poll a barrier; with
+    // two issuers one polls while the other's instructions are queued.
     if (lane == 0) {
-      const int hf = warp - 1;
+      const int iw = warp - 1;
       const uint32_t idesc = make_idesc(kTile, kTile, a.bf16 != 0);
-      int n_item = 0, n_stream = 0, cnt = 0;
+      int n_item = 0, n_stream = 0, cnt[2] = {0, 0};
       bool ok = true;
       while (ok) {
         const int slot = n_item & 1;
@@ -261,25 +261,27 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         ok = mbar_wait(smem_u32(&aux->fixed_full), n_item & 1, abort_flag);
         for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
           const int rs = n_stream % kRing;
-          // also when this half skips the tile: the wait keeps the issuer from running a whole ring ahead of
+          // also when its quarters skip the tile: the wait keeps the issuer from running a whole ring ahead of
           // the other one, whose arrival on empty[rs] must fall into the same phase as this one's
           ok = mbar_wait(smem_u32(&aux->full[rs]), (n_stream / kRing) & 1, abort_flag);
           if (!ok) break;
-          if (g.active(hf, i)) {
-            const int c = cnt++;
-            const int buf = 2 * hf + (c & 1);
-            ok = mbar_wait(smem_u32(&aux->acc_empty[buf]), ((c >> 1) & 1) ^ 1, abort_flag);
+          for (int u = 0; ok && u < 2; ++u) {
+            const int qd = 2 * iw + u;
+            if (!g.active(qd, i)) continue;
+            const int c = cnt[u]++;                 // the quarter's accumulator is reused every time: phase c & 1
+            ok = mbar_wait(smem_u32(&aux->acc_empty[qd]), (c & 1) ^ 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + buf * kTile;
+            const uint32_t d_tmem = tmem_base + qd * kTile;
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
               const uint32_t off = (k >> 2) * SL::kBlockBytes + (k & 3) * 32;
-              umma_bf16(d_tmem, smem_desc_sw128(fixed_addr + hf * SL::kTileBytes + off),
+              umma_bf16(d_tmem, smem_desc_sw128(fixed_addr + qd * SL::kTileBytes + off),
                         smem_desc_sw128(ring_addr + rs * SL::kTileBytes + off), idesc, k > 0);
             }
-            umma_commit(smem_u32(&aux->acc_full[buf]));
+            umma_commit(smem_u32(&aux->acc_full[qd]));
           }
+          if (!ok) break;
           // this issuer is done with the ring slot (a commit with nothing pending arrives at once)
           umma_commit(smem_u32(&aux->empty[rs]));
         }
@@ -289,14 +291,13 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       if (*abort_flag) {
         // wait (bounded) until every MMA already issued has retired before TMEM and shared memory go away
-        umma_commit(smem_u32(&aux->drain[hf]));
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->drain[hf]), 0); ++i) {}
+        umma_commit(smem_u32(&aux->drain[iw]));
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->drain[iw]), 0); ++i) {}
       }
     }
   } else {
     // ------------------------------ epilogue groups ------------------------------
-    const int gi = (warp - 1 - kIssueWarps) >> 2;  // group = half * 2 + parity
-    const int hf = gi >> 1, par = gi & 1;
+    const int gi = (warp - 1 - kIssueWarps) >> 2;  // group = stationary quarter; it owns that quarter's accumulator
     const int quarter = warp & 3;                  // TMEM lanes this warp may read
     const int r = quarter * 32 + lane;             // row of the accumulator = TMEM lane = index inside the group
     const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + gi * kTile;
@@ -304,23 +305,17 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const float scale = a.scale_log2;
     const f32x2 scale2 = splat2(scale);
     const float ninf = __int_as_float(0xFF800000);
-    int n_item = 0, cnt = 0, n_gsync = 0, n_psync = 0;
+    int n_item = 0, cnt = 0, n_gsync = 0;
     bool ok = true;
 
-    // barrier among the 4 warps of the group / the 8 warps of the half; bounded like every other wait
+    // barrier among the 4 warps of the group; bounded like every other wait
     auto group_sync = [&]() {
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&aux->group_bar[gi]));
       ok = mbar_wait(smem_u32(&aux->group_bar[gi]), n_gsync & 1, abort_flag) && ok;
       ++n_gsync;
     };
-    auto pair_sync = [&]() {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&aux->pair_bar[hf]));
-      ok = mbar_wait(smem_u32(&aux->pair_bar[hf]), n_psync & 1, abort_flag) && ok;
-      ++n_psync;
-    };
-    auto release = [&]() {                         // accumulator drained: hand it back to the MMA warp
+    auto release = [&]() {                         // accumulator drained: hand it back to its issuer
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty);
@@ -338,7 +333,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (lane == 0) mbar_arrive(smem_u32(&aux->item_empty[slot]));
       if (it[0] < 0) break;
       const Geo<kColsum> g(s, it);
-      const int row = g.blk * kBlockRows + hf * kTile + r;          // token of this thread inside the sequence
+      const int row = g.blk * kBlockRows + gi * kTile + r;          // token of this thread inside the sequence
       const size_t out = ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0 + row;
 
       if constexpr (kColsum) {
@@ -348,25 +343,22 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           return (i < g.n_iter && j < g.L && j >= g.ws) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
         };
         f32x2 acc[2] = {0ull, 0ull};
-        // this group's tiles of the item: every other active tile, starting where the running parity says
-        int first = g.causal ? max(0, 2 * g.blk + hf - g.first_stream) : 0;
-        if (((cnt & 1) != par)) ++first;
+        int first = g.causal ? max(0, kQ * g.blk + gi - g.first_stream) : 0;    // first tile active for this quarter
         float lse_next = load_lse(first);
         int n_mine = 0;
         for (int i = 0; i < g.n_iter && ok; ++i) {
-          if (!g.active(hf, i)) continue;
+          if (!g.active(gi, i)) continue;
           const int c = cnt++;
-          if ((c & 1) != par) continue;
           float* lse_buf = aux->lse_sh[gi][n_mine & 1];
           ++n_mine;
           lse_buf[r] = lse_next;
-          lse_next = load_lse(i + 2);               // in flight while this tile is processed
+          lse_next = load_lse(i + 1);               // in flight while this tile is processed
           group_sync();
-          ok = mbar_wait(acc_full, (c >> 1) & 1, abort_flag) && ok;
+          ok = mbar_wait(acc_full, c & 1, abort_flag) && ok;
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
           tc_fence_after();
-          if (g.diag(hf, i))
+          if (g.diag(gi, i))
             sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
           else
             sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
@@ -374,13 +366,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         float total = sum4(acc);
-        float* part = aux->part[hf][n_item & 1][0];
-        if (par == 1) part[r] = total;
-        pair_sync();
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-        if (par == 0 && row < g.L && (hf == 0 || g.half1)) {
-          total += part[r];
+        if (row < g.L) {
           if (a.normalize) total = total / (float)(g.L - g.ws);
           a.scores[out] = total;
         }
@@ -388,15 +374,14 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         float m = __int_as_float(0xFF800000);                   // running max (log2 domain) of this row
         f32x2 sum2[2] = {0ull, 0ull};                           // packed partial sums of 2^(x - m)
         for (int i = 0; i < g.n_iter && ok; ++i) {
-          if (!g.active(hf, i)) continue;
+          if (!g.active(gi, i)) continue;
           const int c = cnt++;
-          if ((c & 1) != par) continue;
-          ok = mbar_wait(acc_full, (c >> 1) & 1, abort_flag) && ok;
+          ok = mbar_wait(acc_full, c & 1, abort_flag) && ok;
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
           tc_fence_after();
           // keys of this tile that count for this row: up to the diagonal (causal) and inside the sequence
-          const int n_valid = g.causal ? (g.diag(hf, i) ? r + 1 : kTile) : min(kTile, g.L - i * kTile);
+          const int n_valid = g.causal ? (g.diag(gi, i) ? r + 1 : kTile) : min(kTile, g.L - i * kTile);
           if (__any_sync(0xFFFFFFFFu, n_valid < kTile))
             sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, scale2, n_valid - p * 16, m, sum2); }, release);
           else
@@ -405,17 +390,8 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         const float sum = sum4(sum2);
-        float* pm = aux->part[hf][n_item & 1][0];
-        float* ps = aux->part[hf][n_item & 1][1];
-        if (par == 1) { pm[r] = m; ps[r] = sum; }
-        pair_sync();
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-        if (par == 0 && row < g.L && row >= g.ws && (hf == 0 || g.half1)) {   // merge the other group's (max, sum)
-          const float m1 = pm[r], sum1 = ps[r];
-          const float big = fmaxf(m, m1);
-          const float tot = (sum > 0.f ? sum * ex2(m - big) : 0.f) + (sum1 > 0.f ? sum1 * ex2(m1 - big) : 0.f);
-          const float lse2 = big + log2f(tot);
+        if (row < g.L && row >= g.ws) {
+          const float lse2 = m + log2f(sum);
           a.lse2_out[out] = lse2;
           if (a.lse_nat_out) a.lse_nat_out[out] = lse2 * 0.69314718055994530942f;
         }
