@@ -143,10 +143,11 @@ __device__ __forceinline__ f32x2 exp2_poly2(f32x2 x) {
 }
 
 // Share of the exponentials that takes the FMA-pipe path, in pairs out of every 4 pairs, per sweep.
-// Measured under the board power limit (32 layers x 32 heads x 8192 tokens): the row sweep is fastest
-// with none, the column sweep with one pair in four.
+// Measured at the board power limit (32 layers x 32 heads x 8192 tokens, loops of several seconds): one pair in
+// four is the best share for both sweeps; none costs cycles (the special-function unit saturates), two cost more
+// instructions and energy than they save.
 #ifndef KVC_POLY_PAIRS_LSE
-#define KVC_POLY_PAIRS_LSE 0
+#define KVC_POLY_PAIRS_LSE 1
 #endif
 #ifndef KVC_POLY_PAIRS_COLSUM
 #define KVC_POLY_PAIRS_COLSUM 1
