@@ -74,7 +74,7 @@ struct PSmem {
   static constexpr int kFixedOff = 0;                            // the stationary quarters
   static constexpr int kRingOff = kQ * kTileBytes;
   static constexpr int kAuxOff = kRingOff + kRing * kTileBytes;
-  static constexpr int kAuxBytes = 10240;
+  static constexpr int kAuxBytes = 14336;
   static constexpr int kTotal = kAuxOff + kAuxBytes + 1024;
 };
 
@@ -84,11 +84,13 @@ struct PAux {
   unsigned long long acc_full[kQ], acc_empty[kQ];     // [quarter]
   unsigned long long item_full[2], item_empty[2];
   unsigned long long group_bar[kQ];                   // one epilogue group (4 warps)
+  unsigned long long epi_bar;                         // all epilogue warps (sweep 1 with an observation window)
   unsigned long long drain[kIssueWarps];
   uint32_t tmem_base;
   int abort_flag;
   int item[2][8];                                     // layer, head, seq, block, n_tiles (layer < 0: no more work)
   alignas(16) float lse_sh[kQ][2][kTile];             // [group][buffer][query of the streamed tile]
+  alignas(16) float part[2][kQ][2][kTile];            // [item parity][slot][max, sum][row]: sweep 1, replicated quarters
 };
 
 // Geometry of one work item, derived identically by every role.
@@ -98,6 +100,10 @@ struct Geo {
   int ws;                      // first query row that votes (0 without an observation window)
   bool causal;
   int nq;                      // quarters of the block that hold rows of the sequence
+  // The four accumulator slots normally hold the four quarters.  In sweep 1 with an observation window only the
+  // quarters with voting queries have work; when these are one or two, each is loaded into rep = 4 or 2 slots and
+  // slot s takes the streamed tiles it with it % rep == s % rep, so that all four epilogue groups stay busy.
+  int rep, v0;                 // slots per voting quarter; first voting quarter
   __device__ __forceinline__ Geo(const Shape& s, const int* it) {
     layer = it[0]; h = it[1]; hk = h / s.G; blk = it[3];
     const int seq = it[2], n_tiles = it[4];
@@ -106,22 +112,29 @@ struct Geo {
     causal = s.causal != 0;
     nq = min(kQ, (L - blk * kBlockRows + kTile - 1) / kTile);
     ws = (s.window > 0 && L > s.window) ? L - s.window : 0;
+    rep = 1; v0 = 0;
     if (kColsum) {                                                      // stationary keys, streamed query tiles
       first_stream = max(causal ? kQ * blk : 0, ws / kTile);
       n_iter = n_tiles - first_stream;
     } else {                                                            // stationary queries, streamed key tiles
       first_stream = 0;
       n_iter = causal ? min(kQ * blk + kQ, n_tiles) : n_tiles;
+      if (ws > blk * kBlockRows) v0 = min(nq - 1, (ws - blk * kBlockRows) / kTile);
+      if (s.window > 0) rep = nq - v0 == 1 ? 4 : (nq - v0 == 2 ? 2 : 1);
     }
   }
-  // does streamed tile `it` contribute to quarter `qd` (causal: the quarter's own tile index is kQ*blk + qd)
-  __device__ __forceinline__ bool active(int qd, int it) const {
-    if (qd >= nq) return false;
-    if (!kColsum && blk * kBlockRows + qd * kTile + kTile <= ws) return false;   // no query of this quarter votes
+  __device__ __forceinline__ int n_slots() const { return rep > 1 ? kQ : nq; }
+  __device__ __forceinline__ int quarter(int slot) const { return rep > 1 ? v0 + slot / rep : slot; }
+  // does streamed tile `it` contribute to slot `sl` (causal: the quarter's own tile index is kQ*blk + quarter)
+  __device__ __forceinline__ bool active(int sl, int it) const {
+    const int qd = quarter(sl);
+    if (qd >= nq || qd < v0) return false;                              // no rows, or no voting query
+    if (rep > 1 && it % rep != sl % rep) return false;
     if (!causal) return true;
     return kColsum ? first_stream + it >= kQ * blk + qd : it <= kQ * blk + qd;
   }
-  __device__ __forceinline__ bool diag(int qd, int it) const {
+  __device__ __forceinline__ bool diag(int sl, int it) const {
+    const int qd = quarter(sl);
     return causal && (kColsum ? first_stream + it == kQ * blk + qd : it == kQ * blk + qd);
   }
 };
@@ -153,6 +166,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         mbar_init(smem_u32(&aux->acc_empty[i]), 4);
         mbar_init(smem_u32(&aux->group_bar[i]), 4);
       }
+      mbar_init(smem_u32(&aux->epi_bar), kEpiWarps);
       for (int i = 0; i < 2; ++i) {
         mbar_init(smem_u32(&aux->item_full[i]), 1);
         mbar_init(smem_u32(&aux->item_empty[i]), kIssueWarps + kEpiWarps);
@@ -208,12 +222,13 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // the stationary buffer is free once every MMA of the previous item has retired
         ok = mbar_wait(smem_u32(&aux->fixed_empty), (n_item & 1) ^ 1, abort_flag);
         if (ok) {
-          mbar_expect_tx(smem_u32(&aux->fixed_full), g.nq * SL::kTileBytes);
-          for (int hf = 0; hf < g.nq; ++hf)
+          const int n_slots = g.n_slots();
+          mbar_expect_tx(smem_u32(&aux->fixed_full), n_slots * SL::kTileBytes);
+          for (int sl = 0; sl < n_slots; ++sl)
 #pragma unroll
             for (int kb = 0; kb < D / 64; ++kb)
-              tma_load_4d(fixed_addr + hf * SL::kTileBytes + kb * SL::kBlockBytes, map_fixed, smem_u32(&aux->fixed_full),
-                          kb * 64, g.t0 + g.blk * kBlockRows + hf * kTile, head_fixed, g.layer);
+              tma_load_4d(fixed_addr + sl * SL::kTileBytes + kb * SL::kBlockBytes, map_fixed, smem_u32(&aux->fixed_full),
+                          kb * 64, g.t0 + g.blk * kBlockRows + g.quarter(sl) * kTile, head_fixed, g.layer);
           issued_item = n_item + 1;
           for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
             const int rs = n_stream % kRing;
@@ -305,7 +320,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const float scale = a.scale_log2;
     const f32x2 scale2 = splat2(scale);
     const float ninf = __int_as_float(0xFF800000);
-    int n_item = 0, cnt = 0, n_gsync = 0;
+    int n_item = 0, cnt = 0, n_gsync = 0, n_esync = 0;
     bool ok = true;
 
     // barrier among the 4 warps of the group; bounded like every other wait
@@ -333,7 +348,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (lane == 0) mbar_arrive(smem_u32(&aux->item_empty[slot]));
       if (it[0] < 0) break;
       const Geo<kColsum> g(s, it);
-      const int row = g.blk * kBlockRows + gi * kTile + r;          // token of this thread inside the sequence
+      const int row = g.blk * kBlockRows + g.quarter(gi) * kTile + r;   // token of this thread inside the sequence
       const size_t out = ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0 + row;
 
       if constexpr (kColsum) {
@@ -389,8 +404,31 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
-        const float sum = sum4(sum2);
-        if (row < g.L && row >= g.ws) {
+        float sum = sum4(sum2);
+        if (s.window > 0) {                  // slots that share a quarter merge their (max, sum) through shared memory
+          float* pm = aux->part[n_item & 1][gi][0];
+          float* ps = aux->part[n_item & 1][gi][1];
+          pm[r] = m;
+          ps[r] = sum;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&aux->epi_bar));
+          ok = mbar_wait(smem_u32(&aux->epi_bar), n_esync & 1, abort_flag) && ok;
+          ++n_esync;
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          if (g.rep > 1 && gi % g.rep == 0) {
+            float big = m;
+            for (int u = 1; u < g.rep; ++u) big = fmaxf(big, aux->part[n_item & 1][gi + u][0][r]);
+            float tot = sum > 0.f ? sum * ex2(m - big) : 0.f;
+            for (int u = 1; u < g.rep; ++u) {
+              const float mu = aux->part[n_item & 1][gi + u][0][r], su = aux->part[n_item & 1][gi + u][1][r];
+              tot += su > 0.f ? su * ex2(mu - big) : 0.f;
+            }
+            m = big;
+            sum = tot;
+          }
+        }
+        if (row < g.L && row >= g.ws && (g.rep == 1 || gi % g.rep == 0)) {
           const float lse2 = m + log2f(sum);
           a.lse2_out[out] = lse2;
           if (a.lse_nat_out) a.lse_nat_out[out] = lse2 * 0.69314718055994530942f;
@@ -435,7 +473,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
                                    float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws,
                                    int* counters, float* scores, float* lse_out, int normalize, int32_t* status,
                                    cudaStream_t stream) {
-  static_assert(sizeof(PAux) <= 10240, "aux block too large");
+  static_assert(sizeof(PAux) <= 14336, "aux block too large");
   if (!(scale_log2 > 0.f)) return KVCRUSH_ERR_UNSUPPORTED;
   CUtensorMap mq, mk;
   if (!make_map(&mq, Q, s.D, s.T, s.Hq, s.n_layers) || !make_map(&mk, K, s.D, s.T, s.Hkv, s.n_layers))
