@@ -142,19 +142,19 @@ __device__ __forceinline__ f32x2 exp2_poly2(f32x2 x) {
   return pack2(__float_as_uint(p0) + (__float_as_uint(t0) << 23), __float_as_uint(p1) + (__float_as_uint(t1) << 23));
 }
 
-// Share of the exponentials that takes the FMA-pipe path, in pairs out of every 4 pairs, per sweep.
-// Measured at the board power limit (32 layers x 32 heads x 8192 tokens, loops of several seconds): one pair in
-// four is the best share for both sweeps; none costs cycles (the special-function unit saturates), two cost more
+// Share of the exponentials that takes the FMA-pipe path, in pairs out of every 8 pairs (one 16-column piece), per sweep.
+// Measured at the board power limit (32 layers x 32 heads x 8192 tokens, loops of several seconds): two pairs in
+// eight are the best share for both sweeps; none costs cycles (the special-function unit saturates), two cost more
 // instructions and energy than they save.
 #ifndef KVC_POLY_PAIRS_LSE
-#define KVC_POLY_PAIRS_LSE 1
+#define KVC_POLY_PAIRS_LSE 2
 #endif
 #ifndef KVC_POLY_PAIRS_COLSUM
-#define KVC_POLY_PAIRS_COLSUM 1
+#define KVC_POLY_PAIRS_COLSUM 2
 #endif
 template <int J, int P>
 __device__ __forceinline__ f32x2 exp2_mix2(f32x2 x) {
-  constexpr bool poly = ((J % 4 + 1) * P) / 4 > ((J % 4) * P) / 4;
+  constexpr bool poly = ((J % 8 + 1) * P) / 8 > ((J % 8) * P) / 8;
   if constexpr (poly) return exp2_poly2(x); else return exp2_sfu2(x);
 }
 
@@ -223,10 +223,10 @@ __device__ __forceinline__ void colsum_piece(const uint32_t (&v)[16], const floa
   acc[1] = add2(acc[1], colsum_pair<1, kDiag>(v[2], v[3], la.z, la.w, scale2, r, c0 + 2));
   acc[0] = add2(acc[0], colsum_pair<2, kDiag>(v[4], v[5], lb.x, lb.y, scale2, r, c0 + 4));
   acc[1] = add2(acc[1], colsum_pair<3, kDiag>(v[6], v[7], lb.z, lb.w, scale2, r, c0 + 6));
-  acc[0] = add2(acc[0], colsum_pair<0, kDiag>(v[8], v[9], lc.x, lc.y, scale2, r, c0 + 8));
-  acc[1] = add2(acc[1], colsum_pair<1, kDiag>(v[10], v[11], lc.z, lc.w, scale2, r, c0 + 10));
-  acc[0] = add2(acc[0], colsum_pair<2, kDiag>(v[12], v[13], ld.x, ld.y, scale2, r, c0 + 12));
-  acc[1] = add2(acc[1], colsum_pair<3, kDiag>(v[14], v[15], ld.z, ld.w, scale2, r, c0 + 14));
+  acc[0] = add2(acc[0], colsum_pair<4, kDiag>(v[8], v[9], lc.x, lc.y, scale2, r, c0 + 8));
+  acc[1] = add2(acc[1], colsum_pair<5, kDiag>(v[10], v[11], lc.z, lc.w, scale2, r, c0 + 10));
+  acc[0] = add2(acc[0], colsum_pair<6, kDiag>(v[12], v[13], ld.x, ld.y, scale2, r, c0 + 12));
+  acc[1] = add2(acc[1], colsum_pair<7, kDiag>(v[14], v[15], ld.z, ld.w, scale2, r, c0 + 14));
 }
 
 // ---- sweep 1: 16 columns (keys) of this thread's query row; online max / sum in the log2 domain ----
@@ -260,10 +260,10 @@ __device__ __forceinline__ void lse_piece(const uint32_t (&v)[16], float scale, 
   sum2[1] = add2(sum2[1], exp2_mix2<1, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[2], x[3]), scale2, nm)));
   sum2[0] = add2(sum2[0], exp2_mix2<2, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[4], x[5]), scale2, nm)));
   sum2[1] = add2(sum2[1], exp2_mix2<3, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[6], x[7]), scale2, nm)));
-  sum2[0] = add2(sum2[0], exp2_mix2<0, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[8], x[9]), scale2, nm)));
-  sum2[1] = add2(sum2[1], exp2_mix2<1, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[10], x[11]), scale2, nm)));
-  sum2[0] = add2(sum2[0], exp2_mix2<2, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[12], x[13]), scale2, nm)));
-  sum2[1] = add2(sum2[1], exp2_mix2<3, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[14], x[15]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<4, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[8], x[9]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<5, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[10], x[11]), scale2, nm)));
+  sum2[0] = add2(sum2[0], exp2_mix2<6, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[12], x[13]), scale2, nm)));
+  sum2[1] = add2(sum2[1], exp2_mix2<7, KVC_POLY_PAIRS_LSE>(fma2(pack2(x[14], x[15]), scale2, nm)));
 }
 __device__ __forceinline__ float sum4(const f32x2 (&s)[2]) {
   float a, b, c, d;
