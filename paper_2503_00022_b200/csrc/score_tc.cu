@@ -49,6 +49,7 @@ constexpr int kIssueWarps = 2;                // one tcgen05.mma issuer per stat
 constexpr int kThreads = 32 * (1 + kIssueWarps) + kEpiWarps * 32;
 constexpr int kRing = 2;                     // streamed tiles in flight
 constexpr uint32_t kTmemCols = 512;          // one 128-column fp32 accumulator per quarter
+constexpr int kLseChunk = 16;                // sweep 2: streamed tiles whose row log-sum-exp is staged at once
 
 struct PersistArgs {
   Shape s;
@@ -74,7 +75,7 @@ struct PSmem {
   static constexpr int kFixedOff = 0;                            // the stationary quarters
   static constexpr int kRingOff = kQ * kTileBytes;
   static constexpr int kAuxOff = kRingOff + kRing * kTileBytes;
-  static constexpr int kAuxBytes = 14336;
+  static constexpr int kAuxBytes = 26624;
   static constexpr int kTotal = kAuxOff + kAuxBytes + 1024;
 };
 
@@ -83,13 +84,13 @@ struct PAux {
   unsigned long long fixed_full, fixed_empty;
   unsigned long long acc_full[kQ], acc_empty[kQ];     // [quarter]
   unsigned long long item_full[2], item_empty[2];
-  unsigned long long group_bar[kQ];                   // one epilogue group (4 warps)
-  unsigned long long epi_bar;                         // all epilogue warps (sweep 1 with an observation window)
+  unsigned long long epi_bar;                         // all epilogue warps (sweep 2: a chunk of -lse2 is in place;
+                                                      // sweep 1 with an observation window: slots merge)
   unsigned long long drain[kIssueWarps];
   uint32_t tmem_base;
   int abort_flag;
   int item[2][8];                                     // layer, head, seq, block, n_tiles (layer < 0: no more work)
-  alignas(16) float lse_sh[kQ][2][kTile];             // [group][buffer][query of the streamed tile]
+  alignas(16) float lse_chunk[2][kLseChunk * kTile];  // [buffer][streamed tile inside the chunk][query]: minus lse2
   alignas(16) float part[2][kQ][2][kTile];            // [item parity][slot][max, sum][row]: sweep 1, replicated quarters
 };
 
@@ -164,7 +165,6 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       for (int i = 0; i < kQ; ++i) {
         mbar_init(smem_u32(&aux->acc_full[i]), 1);
         mbar_init(smem_u32(&aux->acc_empty[i]), 4);
-        mbar_init(smem_u32(&aux->group_bar[i]), 4);
       }
       mbar_init(smem_u32(&aux->epi_bar), kEpiWarps);
       for (int i = 0; i < 2; ++i) {
@@ -320,15 +320,15 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const float scale = a.scale_log2;
     const f32x2 scale2 = splat2(scale);
     const float ninf = __int_as_float(0xFF800000);
-    int n_item = 0, cnt = 0, n_gsync = 0, n_esync = 0;
+    int n_item = 0, cnt = 0, n_esync = 0;
     bool ok = true;
 
-    // barrier among the 4 warps of the group; bounded like every other wait
-    auto group_sync = [&]() {
+    // barrier among all 16 epilogue warps; bounded like every other wait
+    auto epi_sync = [&]() {
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&aux->group_bar[gi]));
-      ok = mbar_wait(smem_u32(&aux->group_bar[gi]), n_gsync & 1, abort_flag) && ok;
-      ++n_gsync;
+      if (lane == 0) mbar_arrive(smem_u32(&aux->epi_bar));
+      ok = mbar_wait(smem_u32(&aux->epi_bar), n_esync & 1, abort_flag) && ok;
+      ++n_esync;
     };
     auto release = [&]() {                         // accumulator drained: hand it back to its issuer
       tc_fence_before();
@@ -353,30 +353,41 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
       if constexpr (kColsum) {
         const float* lse_row = a.lse + ((size_t)g.layer * s.Hq + g.h) * s.T + g.t0;
-        auto load_lse = [&](int i) {                // minus lse2 of this thread's query of streamed tile i (-inf past the end)
-          const int j = (g.first_stream + i) * kTile + r;
-          return (i < g.n_iter && j < g.L && j >= g.ws) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
+        // Minus lse2 of the streamed queries reaches the epilogue threads through shared memory, kLseChunk tiles
+        // at a time and once for all four groups: all 16 warps fill the next chunk's buffer, then work through the
+        // current chunk, and meet once per chunk (the buffer of chunk k is rewritten as chunk k + 2 only after
+        // everybody left chunk k).
+        const int et = tid - 32 * (1 + kIssueWarps);
+        auto fill = [&](int k) {
+          float* dst = aux->lse_chunk[k & 1];
+#pragma unroll
+          for (int e = et; e < kLseChunk * kTile; e += kEpiWarps * 32) {
+            const int i = kLseChunk * k + (e >> 7);
+            const int j = (g.first_stream + i) * kTile + (e & (kTile - 1));
+            dst[e] = (i < g.n_iter && j < g.L && j >= g.ws) ? -(__ldg(lse_row + j) * a.lse_mul) : ninf;
+          }
         };
         f32x2 acc[2] = {0ull, 0ull};
-        int first = g.causal ? max(0, kQ * g.blk + gi - g.first_stream) : 0;    // first tile active for this quarter
-        float lse_next = load_lse(first);
-        int n_mine = 0;
-        for (int i = 0; i < g.n_iter && ok; ++i) {
-          if (!g.active(gi, i)) continue;
-          const int c = cnt++;
-          float* lse_buf = aux->lse_sh[gi][n_mine & 1];
-          ++n_mine;
-          lse_buf[r] = lse_next;
-          lse_next = load_lse(i + 1);               // in flight while this tile is processed
-          group_sync();
-          ok = mbar_wait(acc_full, c & 1, abort_flag) && ok;
-          ok = __all_sync(0xFFFFFFFFu, ok);
-          if (!ok) break;
-          tc_fence_after();
-          if (g.diag(gi, i))
-            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
-          else
-            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
+        const int n_chunks = (g.n_iter + kLseChunk - 1) / kLseChunk;
+        fill(0);
+        epi_sync();
+        for (int k = 0; k < n_chunks && ok; ++k) {
+          if (k + 1 < n_chunks) fill(k + 1);
+          const int i_end = min(g.n_iter, kLseChunk * (k + 1));
+          for (int i = kLseChunk * k; i < i_end && ok; ++i) {
+            if (!g.active(gi, i)) continue;
+            const int c = cnt++;
+            const float* lse_buf = aux->lse_chunk[k & 1] + (i & (kLseChunk - 1)) * kTile;
+            ok = mbar_wait(acc_full, c & 1, abort_flag) && ok;
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            if (g.diag(gi, i))
+              sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
+            else
+              sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
+          }
+          epi_sync();
         }
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
@@ -410,10 +421,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           float* ps = aux->part[n_item & 1][gi][1];
           pm[r] = m;
           ps[r] = sum;
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&aux->epi_bar));
-          ok = mbar_wait(smem_u32(&aux->epi_bar), n_esync & 1, abort_flag) && ok;
-          ++n_esync;
+          epi_sync();
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
           if (g.rep > 1 && gi % g.rep == 0) {
@@ -473,7 +481,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
                                    float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws,
                                    int* counters, float* scores, float* lse_out, int normalize, int32_t* status,
                                    cudaStream_t stream) {
-  static_assert(sizeof(PAux) <= 14336, "aux block too large");
+  static_assert(sizeof(PAux) <= 26624, "aux block too large");
   if (!(scale_log2 > 0.f)) return KVCRUSH_ERR_UNSUPPORTED;
   CUtensorMap mq, mk;
   if (!make_map(&mq, Q, s.D, s.T, s.Hq, s.n_layers) || !make_map(&mk, K, s.D, s.T, s.Hkv, s.n_layers))
