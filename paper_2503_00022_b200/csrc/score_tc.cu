@@ -45,7 +45,11 @@ constexpr int kTile = 128;
 constexpr int kQ = 4;                        // stationary 128-row quarters per work item
 constexpr int kBlockRows = kQ * kTile;       // stationary rows per work item
 constexpr int kEpiWarps = 16;
-constexpr int kIssueWarps = 2;                // one tcgen05.mma issuer per stationary half
+#ifndef KVC_ISSUE_WARPS
+#define KVC_ISSUE_WARPS 2
+#endif
+constexpr int kIssueWarps = KVC_ISSUE_WARPS;   // tcgen05.mma issuing threads; each owns kQ / kIssueWarps quarters
+constexpr int kQPerIssuer = kQ / kIssueWarps;
 constexpr int kThreads = 32 * (1 + kIssueWarps) + kEpiWarps * 32;
 constexpr int kRing = 2;                     // streamed tiles in flight
 constexpr uint32_t kTmemCols = 512;          // one 128-column fp32 accumulator per quarter
@@ -261,7 +265,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (lane == 0) {
       const int iw = warp - 1;
       const uint32_t idesc = make_idesc(kTile, kTile, a.bf16 != 0);
-      int n_item = 0, n_stream = 0, cnt[2] = {0, 0};
+      int n_item = 0, n_stream = 0, cnt[kQPerIssuer] = {};
       bool ok = true;
       while (ok) {
         const int slot = n_item & 1;
@@ -280,8 +284,10 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // the other one, whose arrival on empty[rs] must fall into the same phase as this one's
           ok = mbar_wait(smem_u32(&aux->full[rs]), (n_stream / kRing) & 1, abort_flag);
           if (!ok) break;
-          for (int u = 0; ok && u < 2; ++u) {
-            const int qd = 2 * iw + u;
+#pragma unroll
+          for (int u = 0; u < kQPerIssuer; ++u) {
+            if (!ok) break;
+            const int qd = kQPerIssuer * iw + u;
             if (!g.active(qd, i)) continue;
             const int c = cnt[u]++;                 // the quarter's accumulator is reused every time: phase c & 1
             ok = mbar_wait(smem_u32(&aux->acc_empty[qd]), (c & 1) ^ 1, abort_flag);
