@@ -157,3 +157,30 @@ def test_head_dims_between_the_kernel_widths(B, D):
         a, b = int(cu[s_]), int(cu[s_ + 1])
         c, _ = O.scores(inputs.widen(lis[0].q[a:b], w.qk_dtype), inputs.widen(lis[0].k[a:b], w.qk_dtype), True)
         assert TL.within_score_tolerance(got[0][:, a:b], c).all(), (D, s_)
+
+
+def test_logit_jumps_of_hundreds_between_tiles(B):
+    """Keys whose norm jumps by 60x after the first tiles: the row maximum moves by hundreds (log2 domain) between tiles, far beyond what a stale reference can absorb, so the row sweep has to fall back to exact
+    maxima; later tiles fall back again and again as the norm keeps growing."""
+    import torch
+    dev = torch.device("cuda:0")
+    w = inputs.Workload("jump", 1, 2, 2, 128, (1500,), inputs.BF16, inputs.BF16, 0.25, base_seed=123)
+    lis, q, k, _, _ = TL.stack_layers(w, range(1), with_cache=False)
+    kf = inputs.widen(k[0], w.qk_dtype).astype(np.float32)
+    kf[200:] *= 60.0
+    kf[700:] *= 4.0
+    kf[1300:] *= 0.001
+    k2 = inputs.to_storage(kf, w.qk_dtype)[None]
+    prob = B.Problem(1, 2, 2, 128, w.seqlens, device=dev)
+    ws = torch.empty(B.kvcrush_workspace_size(prob, B.STAGE_SCORE), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    c, _ = O.scores(inputs.widen(q[0], w.qk_dtype), inputs.widen(k2[0], w.qk_dtype), True)
+    for impl in (B.SCORE_TENSOR, B.SCORE_SIMT):
+        sc = torch.empty((1, 2, 1500), dtype=torch.float32, device=dev)
+        B.kvcrush_score(prob, TL.torch_storage(q, w.qk_dtype, dev), TL.torch_storage(k2, w.qk_dtype, dev), sc,
+                        impl=impl, workspace=ws, status=status)
+        torch.cuda.synchronize()
+        g = sc.cpu().numpy()[0]
+        assert np.isfinite(g).all()
+        ok = TL.within_score_tolerance(g, c)
+        assert ok.all(), (impl, np.argwhere(~ok)[:4], g[~ok][:4], c[~ok][:4])
