@@ -160,8 +160,8 @@ def test_head_dims_between_the_kernel_widths(B, D):
 
 
 def test_logit_jumps_of_hundreds_between_tiles(B):
-    """Keys whose norm jumps by 60x after the first tiles: the row maximum moves by hundreds (log2 domain) between tiles, far beyond what a stale reference can absorb, so the row sweep has to fall back to exact
-    maxima; later tiles fall back again and again as the norm keeps growing."""
+    """Keys whose norm jumps by 60x after the first tiles: the row maximum moves by hundreds (log2 domain) between
+    tiles, and every running sum is rescaled by factors far below the smallest normal number."""
     import torch
     dev = torch.device("cuda:0")
     w = inputs.Workload("jump", 1, 2, 2, 128, (1500,), inputs.BF16, inputs.BF16, 0.25, base_seed=123)
