@@ -414,10 +414,11 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           tc_fence_after();
           // keys of this tile that count for this row: up to the diagonal (causal) and inside the sequence
           const int n_valid = g.causal ? (g.diag(gi, i) ? r + 1 : kTile) : min(kTile, g.L - i * kTile);
-          if (__any_sync(0xFFFFFFFFu, n_valid < kTile))
+          // masked columns, or a row that has no reference yet (its first tile): exact maxima, piece by piece
+          if (__any_sync(0xFFFFFFFFu, n_valid < kTile || !(m > -3.0e38f)))
             sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, scale2, n_valid - p * 16, m, sum2); }, release);
           else
-            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<false>(v, scale, scale2, 16, m, sum2); }, release);
+            lse_tile_lazy(t_acc, scale, scale2, m, sum2, release);
         }
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace kvc {
@@ -270,6 +272,81 @@ __device__ __forceinline__ float sum4(const f32x2 (&s)[2]) {
   unpack2(s[0], a, b);
   unpack2(s[1], c, d);
   return (a + b) + (c + d);
+}
+
+// The same 16 columns added with the reference m left as it is (no maximum is taken): correct as long as no
+// 2^(x - m) overflows.  The special-function unit returns +inf then, which the caller's range check sees in the
+// sums; the polynomial path would wrap around instead, so the largest argument that went through it is tracked.
+__device__ __forceinline__ void lse_piece_lazy(const uint32_t (&x)[16], f32x2 scale2, float m, f32x2 (&sum2)[2],
+                                               float& poly_max) {
+  const f32x2 nm = splat2(-m);
+  auto term = [&](auto jc, uint32_t a, uint32_t b) {
+    constexpr int J = decltype(jc)::value;
+    constexpr bool poly = ((J % 8 + 1) * KVC_POLY_PAIRS_LSE) / 8 > ((J % 8) * KVC_POLY_PAIRS_LSE) / 8;
+    const f32x2 arg = fma2(pack2(a, b), scale2, nm);
+    if constexpr (poly) {
+      float a0, a1;
+      unpack2(arg, a0, a1);
+      poly_max = max3(poly_max, a0, a1);
+      return exp2_poly2(arg);
+    } else {
+      return exp2_sfu2(arg);
+    }
+  };
+  sum2[0] = add2(sum2[0], term(std::integral_constant<int, 0>{}, x[0], x[1]));
+  sum2[1] = add2(sum2[1], term(std::integral_constant<int, 1>{}, x[2], x[3]));
+  sum2[0] = add2(sum2[0], term(std::integral_constant<int, 2>{}, x[4], x[5]));
+  sum2[1] = add2(sum2[1], term(std::integral_constant<int, 3>{}, x[6], x[7]));
+  sum2[0] = add2(sum2[0], term(std::integral_constant<int, 4>{}, x[8], x[9]));
+  sum2[1] = add2(sum2[1], term(std::integral_constant<int, 5>{}, x[10], x[11]));
+  sum2[0] = add2(sum2[0], term(std::integral_constant<int, 6>{}, x[12], x[13]));
+  sum2[1] = add2(sum2[1], term(std::integral_constant<int, 7>{}, x[14], x[15]));
+}
+
+// Sweep 1, one whole accumulator (128 unmasked columns) for a row whose reference m is already finite.  The maximum
+// of a softmax row rarely moves after its first tile, and the running sum may use any reference that keeps
+// 2^(x - m) finite, so the first seven pieces are added against the reference as it stands, without the max tree.
+// Before the accumulator is handed back the sums are checked: if any lane of the warp left the range, those pieces
+// are redone exactly from TMEM; a sum that has grown past 2^60 moves the reference up by 60.  The last piece is
+// already in registers and is added exactly.
+template <class Release>
+__device__ __forceinline__ void lse_tile_lazy(uint32_t taddr, float scale, f32x2 scale2, float& m, f32x2 (&sum2)[2],
+                                              Release&& release) {
+  uint32_t va[16], vb[16];
+  const f32x2 keep0 = sum2[0], keep1 = sum2[1];
+  float poly_max = 0.f;
+  tmem_ld16(taddr, va);
+  tmem_wait16(va);
+#pragma unroll
+  for (int p = 0; p < 6; p += 2) {
+    tmem_ld16(taddr + (p + 1) * 16, vb);
+    lse_piece_lazy(va, scale2, m, sum2, poly_max);
+    tmem_wait16(vb);
+    tmem_ld16(taddr + (p + 2) * 16, va);
+    lse_piece_lazy(vb, scale2, m, sum2, poly_max);
+    tmem_wait16(va);
+  }
+  tmem_ld16(taddr + 7 * 16, vb);
+  lse_piece_lazy(va, scale2, m, sum2, poly_max);
+  tmem_wait16(vb);
+  const float total = sum4(sum2);
+  if (__any_sync(0xFFFFFFFFu, !(total < 0x1p100f) || poly_max > 100.f)) {
+    sum2[0] = keep0;
+    sum2[1] = keep1;
+#pragma unroll 1
+    for (int p = 0; p < 7; ++p) {
+      tmem_ld16(taddr + p * 16, va);
+      tmem_wait16(va);
+      lse_piece<false>(va, scale, scale2, 16, m, sum2);
+    }
+  } else if (total > 0x1p60f) {
+    m += 60.f;
+    const f32x2 down = splat2(0x1p-60f);
+    sum2[0] = mul2(sum2[0], down);
+    sum2[1] = mul2(sum2[1], down);
+  }
+  release();
+  lse_piece<false>(vb, scale, scale2, 16, m, sum2);
 }
 
 // Shared-memory matrix descriptor of a K-major tile stored as 128-byte rows with the 128B swizzle
