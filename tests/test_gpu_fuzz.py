@@ -184,3 +184,35 @@ def test_logit_jumps_of_hundreds_between_tiles(B):
         assert np.isfinite(g).all()
         ok = TL.within_score_tolerance(g, c)
         assert ok.all(), (impl, np.argwhere(~ok)[:4], g[~ok][:4], c[~ok][:4])
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_random_key_norm_profiles(B, seed):
+    """Key norms that change by random factors between 1e-2 and 1e2 from one block of 64 tokens to the next, queries
+    likewise: row maxima move up and down by arbitrary amounts from tile to tile."""
+    import torch
+    dev = torch.device("cuda:0")
+    g = np.random.Generator(np.random.Philox(900 + seed))
+    L = int(g.choice([1111, 1664, 2049]))
+    w = inputs.Workload("norms", 1, 4, 2, 128, (L,), inputs.BF16, inputs.BF16, 0.25, base_seed=500 + seed)
+    lis, q, k, _, _ = TL.stack_layers(w, range(1), with_cache=False)
+    qf = inputs.widen(q[0], w.qk_dtype).astype(np.float32)
+    kf = inputs.widen(k[0], w.qk_dtype).astype(np.float32)
+    for a in range(0, L, 64):
+        kf[a:a + 64] *= np.float32(10.0 ** g.uniform(-2, 2))
+        qf[a:a + 64] *= np.float32(10.0 ** g.uniform(-1, 1))
+    q2, k2 = inputs.to_storage(qf, w.qk_dtype)[None], inputs.to_storage(kf, w.qk_dtype)[None]
+    prob = B.Problem(1, 4, 2, 128, w.seqlens, device=dev)
+    ws = torch.empty(B.kvcrush_workspace_size(prob, B.STAGE_SCORE), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    c, lse = O.scores(inputs.widen(q2[0], w.qk_dtype), inputs.widen(k2[0], w.qk_dtype), True)
+    sc = torch.empty((1, 4, L), dtype=torch.float32, device=dev)
+    lo = torch.empty_like(sc)
+    B.kvcrush_score(prob, TL.torch_storage(q2, w.qk_dtype, dev), TL.torch_storage(k2, w.qk_dtype, dev), sc, lse_out=lo,
+                    impl=B.SCORE_TENSOR, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0
+    gl = lo.cpu().numpy()[0]
+    np.testing.assert_allclose(gl, lse, rtol=2e-6, atol=1e-3)
+    ok = TL.within_score_tolerance(sc.cpu().numpy()[0], c)
+    assert ok.all(), (seed, np.argwhere(~ok)[:4])
