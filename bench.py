@@ -34,7 +34,7 @@ from paper_2503_00022_b200 import inputs  # noqa: E402
 METRIC = "prompt tokens compressed/s (score+select+compact)"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg3_llama2_32l_8k"
-NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP = 139e6   # (279.4 + 278.1) MB / 2 sweeps / 2 layers: dram__bytes_read + dram__bytes_write
+NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP = 138.4e6   # (275.5 + 278.2) MB / 2 sweeps / 2 layers: dram__bytes_read + dram__bytes_write
 
 
 def measured_peaks():
@@ -445,7 +445,7 @@ def run_ours(args, w):
     tensor_path = B.lib() is not None and w.qk_dtype == inputs.BF16 and w.head_dim in (64, 128)
     achieved_tf = work["score_flops"] / score_s / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
-    # dram__bytes_read + dram__bytes_write of one sweep launch: 139 MB per layer in the ncu capture of a 2-layer case
+    # dram__bytes_read + dram__bytes_write of one sweep launch: 138 MB per layer in the ncu capture of a 2-layer case
     # of this workload (profiles/score_persist_kernel_cfg3_2layers.md); proportional to the layer count
     traffic = NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP * w.n_layers if (tensor_path and w.name.startswith(DEFAULT_WORKLOAD) and not args.window) else None
     roofline = {"bound": "tensor" if tensor_path else "alu", "kernel": "score_persist_kernel (two sweep launches per step; per-launch figures)" if tensor_path else "score SIMT",
