@@ -57,6 +57,9 @@ because it gives no formula for them:
   the first n tokens (Table 1 splits its 672-token budget into 32 initial + 512 middle +
   128 recent tokens).
 
+Decode step (``decode_update``): the cumulative attention of H2O goes on while tokens are generated; one new query
+adds its softmax row over the cached keys.  PARITY UNPINNED by this paper (it describes the baseline in a sentence).
+
 Chunk- and page-granular eviction (Sec. 4.3.4: chunks of 8 tokens; Sec. 4.3.5: pages of 32 tokens): the
 paper gives two sentences - the baseline sums the attention weights over a page, and the
 binary vector of a page is the concatenation of the head vectors of its tokens.  Everything
@@ -431,6 +434,25 @@ def compact_pages(cache: np.ndarray, page_idx: np.ndarray, page_size: int) -> np
     for i, p in enumerate(np.asarray(page_idx, dtype=np.int64)):
         n = min(page_size, L - int(p) * page_size)
         out[i, :n] = cache[int(p) * page_size:int(p) * page_size + n]
+    return out
+
+
+# ---------------------------------------------------------------------------
+# Decode step of the cumulative attention (Sec. 2.3 / 4.1.1: H2O keeps summing attention weights while decoding)
+# ---------------------------------------------------------------------------
+
+def decode_update(scores: np.ndarray, q_new: np.ndarray, k: np.ndarray, scale: Optional[float] = None) -> np.ndarray:
+    """scores [Hq, L] (float64) plus the attention row of one new query q_new [Hq, D] over all L cached keys
+    k [L, Hkv, D] (the new token's own key is the last one): A_h(t) = softmax_t(q_h . k_t / sqrt(d_k))."""
+    Hq, D = q_new.shape
+    L, Hkv, _ = k.shape
+    G = Hq // Hkv
+    sc = (1.0 / np.sqrt(D)) if scale is None else float(scale)
+    out = np.array(scores, dtype=np.float64, copy=True)
+    for h in range(Hq):
+        logits = (k[:, h // G, :].astype(np.float64) @ q_new[h].astype(np.float64)) * sc
+        e = np.exp(logits - logits.max())
+        out[h] += e / e.sum()
     return out
 
 

@@ -141,3 +141,23 @@ def test_planted_transposition_is_caught():
     # and a dropped causal mask changes the harmonic closed form
     c_nc, _ = O.scores(np.zeros_like(q), k, False)
     assert not np.allclose(c_nc[0], O.scores(np.zeros_like(q), k, True)[0][0])
+
+
+def test_decode_update_adds_the_last_row_of_the_attention_matrix():
+    L, Hq, Hkv, D = 37, 4, 2, 16
+    q, k = _rand_qk(L, Hq, Hkv, D, 31)
+    A = O.attention_matrix(q, k, True)                     # [Hq, query, key]
+    base = np.arange(Hq * L, dtype=np.float64).reshape(Hq, L) / 7.0
+    got = O.decode_update(base, q[L - 1], k)
+    np.testing.assert_allclose(got - base, A[:, L - 1, :], rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose((got - base).sum(axis=1), 1.0, rtol=1e-12)
+    # decoding the whole prompt token by token rebuilds the prefill column sums
+    run = np.zeros((Hq, L))
+    for j in range(L):
+        run[:, : j + 1] = O.decode_update(run[:, : j + 1], q[j], k[: j + 1])
+    c, _ = O.scores(q, k, True)
+    np.testing.assert_allclose(run, c, rtol=1e-11, atol=1e-13)
+    tq = torch.from_numpy(q[L - 1])                        # library softmax
+    tk = torch.from_numpy(k).permute(1, 0, 2).repeat_interleave(Hq // Hkv, dim=0)
+    ref = torch.softmax((tk @ tq[:, :, None])[:, :, 0] / np.sqrt(D), dim=-1).numpy()
+    np.testing.assert_allclose(got - base, ref, rtol=1e-11, atol=1e-14)
