@@ -138,6 +138,23 @@ int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, c
                   void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
 /*
+ * Decode step of stage 1 (Sec. 2.3 / 4.1.1: H2O goes on summing attention weights while tokens are generated, and
+ * the paper's paged experiments evict during decoding).  Every sequence has exactly one new query - the query of its
+ * last token - and
+ *     scores[l][h][t] += softmax over the sequence's tokens of (q_new[l][seq(t)][h] . k[l][t][h div G] * scale)
+ * for every token t of the sequence, the new token included.  Feed the running scores to kvcrush_signature /
+ * kvcrush_select(_pages) whenever the cache has outgrown its budget.
+ *   problem     describes the cached tokens as they are now (cu_seqlens include each sequence's new token);
+ *               causal and query_window are ignored
+ *   Q_new       [n_layers][n_seqs][n_q_heads][head_dim]: stride_token steps from one sequence to the next
+ *   K           the cached keys, token-major, same dtype as Q_new (BF16, FP16 or FP32), head_dim <= 256, multiple of 8
+ *   scores_dev  in/out [n_layers][n_q_heads][T] float32 running column sums
+ * Runs on the CUDA cores (one block per layer, sequence and query head); bound by reading K twice.
+ */
+int kvcrush_score_decode(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q_new, const kvcrush_tensor_t* K,
+                         float* scores_dev, int32_t* status_dev, void* stream);
+
+/*
  * Stage 2 - per-head thresholds and packed signatures (Algorithm 1, Sec. 3.1).
  *   theta[l][s][h] = the keep-th largest value of scores[l][h][tokens of s]
  *                    (keep >= length: -inf, all ones; keep <= 0: +inf, all zeros)

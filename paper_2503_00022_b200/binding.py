@@ -28,7 +28,7 @@ SCORE_AUTO, SCORE_SIMT, SCORE_TENSOR = 0, 1, 2
 
 EXPORTS = ("kvcrush_workspace_size", "kvcrush_score", "kvcrush_signature", "kvcrush_select",
            "kvcrush_compact", "kvcrush_strerror", "kvcrush_version", "kvcrush_signature_static",
-           "kvcrush_pool_scores", "kvcrush_select_pages", "kvcrush_compact_pages")
+           "kvcrush_pool_scores", "kvcrush_select_pages", "kvcrush_compact_pages", "kvcrush_score_decode")
 
 
 class ProblemStruct(ctypes.Structure):
@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
         P, T = ctypes.POINTER(ProblemStruct), ctypes.POINTER(TensorStruct)
         L.kvcrush_workspace_size.argtypes = [P, i32, ctypes.POINTER(sz)]
         L.kvcrush_score.argtypes = [P, T, T, vp, vp, vp, i32, i32, vp, sz, vp, vp]
+        L.kvcrush_score_decode.argtypes = [P, T, T, vp, vp, vp]
         L.kvcrush_signature.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_pool_scores.argtypes = [P, vp, i32, vp, vp, vp]
@@ -157,6 +158,13 @@ def kvcrush_score(problem: Problem, q, k, scores, *, lse_in=None, lse_out=None, 
     _check(lib().kvcrush_score(problem.ref, ctypes.byref(qs), ctypes.byref(ks), _ptr(lse_in), _ptr(scores),
                                _ptr(lse_out), int(normalize), int(impl), _ptr(workspace), ws_bytes, _ptr(status),
                                _stream() if stream is None else stream), "kvcrush_score")
+
+
+def kvcrush_score_decode(problem: Problem, q_new, k, scores, *, status=None, stream: Optional[int] = None) -> None:
+    """Adds the attention row of every sequence's new query (q_new [layers, n_seqs, Hq, D]) to the running scores."""
+    qs, ks = tensor_struct(q_new), tensor_struct(k)
+    _check(lib().kvcrush_score_decode(problem.ref, ctypes.byref(qs), ctypes.byref(ks), _ptr(scores), _ptr(status),
+                                      _stream() if stream is None else stream), "kvcrush_score_decode")
 
 
 def kvcrush_signature(problem: Problem, scores, sigs, *, sig_keep=None, theta_in=None, theta_out=None,

@@ -104,6 +104,20 @@ int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, c
                              scores_dev, lse_out_dev, normalize, status_dev, st);
 }
 
+int kvcrush_score_decode(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q_new, const kvcrush_tensor_t* K,
+                         float* scores_dev, int32_t* status_dev, void* stream) {
+  Shape s;
+  int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  TensorView q, k;
+  if ((rc = make_view(Q_new, s.D, &q)) != KVCRUSH_OK) return rc;
+  if ((rc = make_view(K, s.D, &k)) != KVCRUSH_OK) return rc;
+  if (!scores_dev || !status_dev) return KVCRUSH_ERR_INVALID_ARG;
+  if (q.dtype != k.dtype) return KVCRUSH_ERR_INVALID_ARG;
+  const float scale = problem->softmax_scale != 0.f ? problem->softmax_scale : 1.f / sqrtf((float)s.D);
+  return launch_score_decode(s, q, k, scale * 1.4426950408889634f, scores_dev, static_cast<cudaStream_t>(stream));
+}
+
 int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev, const int32_t* sig_keep_dev,
                       const float* theta_in_dev, uint32_t* sigs_dev, float* theta_out_dev,
                       void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {

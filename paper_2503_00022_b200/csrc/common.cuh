@@ -53,6 +53,9 @@ __device__ __forceinline__ int seq_of_token(const int32_t* __restrict__ cu, int 
 int launch_score_simt(const Shape& s, const TensorView& Q, const TensorView& K, float scale_log2,
                       const float* lse_in, float lse_in_mul, float* lse2_ws, float* scores, float* lse_out,
                       int normalize, int32_t* status, cudaStream_t stream);
+// Decode step: scores[l][h][t] += attention of sequence(t)'s new query (Q_new's token axis = sequence) to key t.
+int launch_score_decode(const Shape& s, const TensorView& Q_new, const TensorView& K, float scale_log2, float* scores,
+                        cudaStream_t stream);
 bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorView& K);
 // `counters`: two ints of caller scratch (work counters of the two persistent sweeps).
 size_t score_tensor_counter_bytes();

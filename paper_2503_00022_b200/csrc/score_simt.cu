@@ -145,6 +145,110 @@ colsum_kernel(Shape s, TensorView Q, TensorView K, float scale_log2, const float
   if (lane == 0) scores[col] = normalize ? acc / (float)(t1 - t0 - ws) : acc;
 }
 
+// Decode step: every sequence has one new query (its last token); the query's attention row over the sequence's
+// cached keys is added to the running scores.  One block per (layer, sequence, KV head); threads stride over the
+// tokens and serve up to kDecodeHeads query heads of the KV group from one read of a key row.  Pass 1 keeps an
+// online (max, sum) per thread and head and reduces it over the block, pass 2 recomputes the logits and adds
+// 2^(x - lse2) to scores (each token is owned by one thread: no atomics).
+constexpr int kDecodeThreads = 256;
+constexpr int kDecodeHeads = 4;
+
+template <typename T>
+__device__ __forceinline__ void dot_rows(const float (*q_sh)[kMaxD], const T* __restrict__ krow, int D, int n_heads,
+                                         float (&acc)[kDecodeHeads]) {
+#pragma unroll
+  for (int g = 0; g < kDecodeHeads; ++g) acc[g] = 0.f;
+  for (int d = 0; d < D; d += 8) {
+    float v[8];
+    load8<T>(krow + d, v);
+#pragma unroll
+    for (int g = 0; g < kDecodeHeads; ++g)
+      if (g < n_heads) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[g] = fmaf(q_sh[g][d + i], v[i], acc[g]);
+      }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kDecodeThreads)
+decode_update_kernel(Shape s, TensorView Qn, TensorView K, float scale_log2, float* __restrict__ scores) {
+  __shared__ float q_sh[kDecodeHeads][kMaxD];
+  __shared__ float red_m[kDecodeHeads][kDecodeThreads / 32], red_s[kDecodeHeads][kDecodeThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, wib = tid >> 5;
+  const int hk = blockIdx.x % s.Hkv;
+  const int seq = (blockIdx.x / s.Hkv) % s.n_seqs;
+  const int layer = blockIdx.x / (s.Hkv * s.n_seqs);
+  const int t0 = __ldg(s.cu_seqlens + seq), t1 = __ldg(s.cu_seqlens + seq + 1);
+  if (t1 <= t0) return;
+  const T* kbase = static_cast<const T*>(K.ptr) + layer * K.sl + hk * K.sh;
+
+  for (int g0 = 0; g0 < s.G; g0 += kDecodeHeads) {                // the KV group's query heads, a few at a time
+    const int n_heads = min(kDecodeHeads, s.G - g0);
+    const int h0 = hk * s.G + g0;
+    __syncthreads();                                              // q_sh / red_* of the previous round are done with
+    for (int e = tid * 8; e < n_heads * s.D; e += kDecodeThreads * 8) {
+      const int g = e / s.D, d = e - g * s.D;
+      const T* q = static_cast<const T*>(Qn.ptr) + layer * Qn.sl + (long long)seq * Qn.st + (h0 + g) * Qn.sh;
+      float v[8];
+      load8<T>(q + d, v);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) q_sh[g][d + i] = v[i];
+    }
+    __syncthreads();
+
+    float m[kDecodeHeads], sum[kDecodeHeads];
+#pragma unroll
+    for (int g = 0; g < kDecodeHeads; ++g) { m[g] = -INFINITY; sum[g] = 0.f; }
+    for (int t = t0 + tid; t < t1; t += kDecodeThreads) {
+      float x[kDecodeHeads];
+      dot_rows<T>(q_sh, kbase + (long long)t * K.st, s.D, n_heads, x);
+#pragma unroll
+      for (int g = 0; g < kDecodeHeads; ++g) {
+        const float xs = x[g] * scale_log2;
+        if (xs > m[g]) { sum[g] = sum[g] * exp2f(m[g] - xs) + 1.f; m[g] = xs; } else { sum[g] += exp2f(xs - m[g]); }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < kDecodeHeads; ++g) {
+      float big = m[g];
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) big = fmaxf(big, __shfl_xor_sync(0xFFFFFFFFu, big, d));
+      float part = (m[g] == -INFINITY) ? 0.f : sum[g] * exp2f(m[g] - big);
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, d);
+      if (lane == 0) { red_m[g][wib] = big; red_s[g][wib] = part; }
+    }
+    __syncthreads();
+    float lse2[kDecodeHeads];
+#pragma unroll
+    for (int g = 0; g < kDecodeHeads; ++g) {
+      float all_m = -INFINITY, all_s = 0.f;
+      for (int w = 0; w < kDecodeThreads / 32; ++w) all_m = fmaxf(all_m, red_m[g][w]);
+      for (int w = 0; w < kDecodeThreads / 32; ++w)
+        all_s += red_m[g][w] == -INFINITY ? 0.f : red_s[g][w] * exp2f(red_m[g][w] - all_m);
+      lse2[g] = all_m + log2f(all_s);
+    }
+
+    for (int t = t0 + tid; t < t1; t += kDecodeThreads) {
+      float x[kDecodeHeads];
+      dot_rows<T>(q_sh, kbase + (long long)t * K.st, s.D, n_heads, x);
+#pragma unroll
+      for (int g = 0; g < kDecodeHeads; ++g)
+        if (g < n_heads) scores[((long long)layer * s.Hq + h0 + g) * s.T + t] += exp2f(x[g] * scale_log2 - lse2[g]);
+    }
+  }
+}
+
+template <typename T>
+int run_decode(const Shape& s, const TensorView& Qn, const TensorView& K, float scale_log2, float* scores,
+               cudaStream_t stream) {
+  const long long blocks = (long long)s.n_layers * s.n_seqs * s.Hkv;
+  if (blocks > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
+  decode_update_kernel<T><<<(unsigned)blocks, kDecodeThreads, 0, stream>>>(s, Qn, K, scale_log2, scores);
+  return check_launch();
+}
+
 template <typename T>
 int run(const Shape& s, const TensorView& Q, const TensorView& K, float scale_log2, const float* lse_in,
         float lse_in_mul, float* lse2_ws, float* scores, float* lse_out, int normalize, cudaStream_t stream) {
@@ -177,6 +281,16 @@ int launch_score_simt(const Shape& s, const TensorView& Q, const TensorView& K, 
     return run<__nv_bfloat16>(s, Q, K, scale_log2, lse_in, lse_in_mul, lse2_ws, scores, lse_out, normalize, stream);
   if (Q.dtype == KVCRUSH_FP16)
     return run<__half>(s, Q, K, scale_log2, lse_in, lse_in_mul, lse2_ws, scores, lse_out, normalize, stream);
+  return KVCRUSH_ERR_UNSUPPORTED;
+}
+
+int launch_score_decode(const Shape& s, const TensorView& Q_new, const TensorView& K, float scale_log2, float* scores,
+                        cudaStream_t stream) {
+  if (s.D > kMaxD || s.D % 8 != 0) return KVCRUSH_ERR_UNSUPPORTED;
+  if (s.T == 0) return KVCRUSH_OK;
+  if (Q_new.dtype == KVCRUSH_FP32) return run_decode<float>(s, Q_new, K, scale_log2, scores, stream);
+  if (Q_new.dtype == KVCRUSH_BF16) return run_decode<__nv_bfloat16>(s, Q_new, K, scale_log2, scores, stream);
+  if (Q_new.dtype == KVCRUSH_FP16) return run_decode<__half>(s, Q_new, K, scale_log2, scores, stream);
   return KVCRUSH_ERR_UNSUPPORTED;
 }
 

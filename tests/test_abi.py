@@ -104,6 +104,10 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
     assert sp(8, prob=long_seq, ws=1 << 30) == B.ERR_UNSUPPORTED
     assert lib.kvcrush_compact_pages(r(p), r(t), None, 0, 0x100, 0x100, 10, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_compact_pages(r(p), r(t), r(t), 8, 0x100, 0x100, 10, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
+    # decode step: NULL scores, dtype mismatch, misaligned tensor
+    assert lib.kvcrush_score_decode(r(p), r(t), r(t), None, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_score_decode(r(p), r(t), r(f16), 0x100, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_score_decode(r(p), r(odd), r(t), 0x100, 0x100, None) == B.ERR_MISALIGNED
     # pooling: even kernel, aliasing
     assert lib.kvcrush_pool_scores(r(p), 0x100, 4, 0x200, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_pool_scores(r(p), 0x100, 3, 0x100, 0x100, None) == B.ERR_INVALID_ARG
