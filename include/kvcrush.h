@@ -272,6 +272,21 @@ int kvcrush_compact_pages(const kvcrush_problem_t* problem, const kvcrush_tensor
                           int32_t* status_dev, void* stream);
 
 /*
+ * The running scores of a decode-time loop follow the cache through an eviction (Sec. 2.3 / 4.1.1: the cumulative
+ * attention of the kept tokens goes on accumulating):
+ *   out[l][h][(cu_kept[l*n_seqs+s] - cu_kept[l*n_seqs] + i) * P + j] = in[l][h][cu_seqlens[s] + idx[cu_kept[..] + i] * P + j]
+ * with P = 1 and j = 0 for kept tokens (page_size 0), P = page_size and j < P for kept pages; slots of a short last
+ * page that lie past the end of the sequence get 0.  The arrangement along the token axis is that of
+ * kvcrush_compact / kvcrush_compact_pages.
+ *   scores_in_dev   [n_layers][n_q_heads][T] float32
+ *   scores_out_dev  out [n_layers][n_q_heads][out_tokens] float32; must not alias the input
+ *   out_tokens      token stride of the output (>= the kept rows of any layer)
+ */
+int kvcrush_compact_scores(const kvcrush_problem_t* problem, const float* scores_in_dev, int page_size,
+                           const int32_t* cu_kept_dev, const int32_t* idx_dev, int64_t total_kept,
+                           float* scores_out_dev, int64_t out_tokens, int32_t* status_dev, void* stream);
+
+/*
  * Stage 2 without caller-provided scratch (the paper has no counterpart; this is a packaging
  * variant of kvcrush_signature for hosts that cannot hand over device memory).
  *

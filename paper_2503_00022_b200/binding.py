@@ -28,7 +28,8 @@ SCORE_AUTO, SCORE_SIMT, SCORE_TENSOR = 0, 1, 2
 
 EXPORTS = ("kvcrush_workspace_size", "kvcrush_score", "kvcrush_signature", "kvcrush_select",
            "kvcrush_compact", "kvcrush_strerror", "kvcrush_version", "kvcrush_signature_static",
-           "kvcrush_pool_scores", "kvcrush_select_pages", "kvcrush_compact_pages", "kvcrush_score_decode")
+           "kvcrush_pool_scores", "kvcrush_select_pages", "kvcrush_compact_pages", "kvcrush_score_decode",
+           "kvcrush_compact_scores")
 
 
 class ProblemStruct(ctypes.Structure):
@@ -69,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.kvcrush_workspace_size.argtypes = [P, i32, ctypes.POINTER(sz)]
         L.kvcrush_score.argtypes = [P, T, T, vp, vp, vp, i32, i32, vp, sz, vp, vp]
         L.kvcrush_score_decode.argtypes = [P, T, T, vp, vp, vp]
+        L.kvcrush_compact_scores.argtypes = [P, vp, i32, vp, vp, i64, vp, i64, vp, vp]
         L.kvcrush_signature.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_pool_scores.argtypes = [P, vp, i32, vp, vp, vp]
@@ -165,6 +167,15 @@ def kvcrush_score_decode(problem: Problem, q_new, k, scores, *, status=None, str
     qs, ks = tensor_struct(q_new), tensor_struct(k)
     _check(lib().kvcrush_score_decode(problem.ref, ctypes.byref(qs), ctypes.byref(ks), _ptr(scores), _ptr(status),
                                       _stream() if stream is None else stream), "kvcrush_score_decode")
+
+
+def kvcrush_compact_scores(problem: Problem, scores_in, page_size: int, cu_kept, idx, total_kept: int, scores_out, *,
+                           status=None, stream: Optional[int] = None) -> None:
+    """Gathers running scores [layers, Hq, T] along the kept tokens (page_size 0) or pages into scores_out
+    [layers, Hq, T_out], arranged like the reduced cache."""
+    _check(lib().kvcrush_compact_scores(problem.ref, _ptr(scores_in), int(page_size), _ptr(cu_kept), _ptr(idx),
+                                        int(total_kept), _ptr(scores_out), int(scores_out.shape[-1]), _ptr(status),
+                                        _stream() if stream is None else stream), "kvcrush_compact_scores")
 
 
 def kvcrush_signature(problem: Problem, scores, sigs, *, sig_keep=None, theta_in=None, theta_out=None,

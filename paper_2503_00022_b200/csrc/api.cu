@@ -235,6 +235,19 @@ int kvcrush_compact_pages(const kvcrush_problem_t* problem, const kvcrush_tensor
                               V ? &vo : nullptr, static_cast<cudaStream_t>(stream));
 }
 
+int kvcrush_compact_scores(const kvcrush_problem_t* problem, const float* scores_in_dev, int page_size,
+                           const int32_t* cu_kept_dev, const int32_t* idx_dev, int64_t total_kept,
+                           float* scores_out_dev, int64_t out_tokens, int32_t* status_dev, void* stream) {
+  Shape s;
+  const int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if (!scores_in_dev || !scores_out_dev || scores_in_dev == scores_out_dev || !cu_kept_dev || !idx_dev || !status_dev)
+    return KVCRUSH_ERR_INVALID_ARG;
+  if (page_size < 0 || total_kept < 0 || out_tokens < 0) return KVCRUSH_ERR_INVALID_ARG;
+  return launch_compact_scores(s, scores_in_dev, page_size, cu_kept_dev, idx_dev, total_kept, scores_out_dev,
+                               out_tokens, static_cast<cudaStream_t>(stream));
+}
+
 int kvcrush_pool_scores(const kvcrush_problem_t* problem, const float* scores_in_dev, int kernel,
                         float* scores_out_dev, int32_t* status_dev, void* stream) {
   Shape s;

@@ -87,6 +87,11 @@ int launch_compact_pages(const Shape& s, const TensorView& K, const TensorView* 
                          const int32_t* cu_kept, const int32_t* page_idx, long long total_kept_pages,
                          const TensorView& K_out, const TensorView* V_out, cudaStream_t stream);
 
+// Gather of the running scores along the kept tokens (page_size 0) or kept pages.
+int launch_compact_scores(const Shape& s, const float* scores_in, int page_size, const int32_t* cu_kept,
+                          const int32_t* idx, long long total_kept, float* scores_out, long long out_tokens,
+                          cudaStream_t stream);
+
 int launch_pool_scores(const Shape& s, const float* scores_in, int kernel, float* scores_out, cudaStream_t stream);
 
 int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, const int32_t* cu_kept,

@@ -89,6 +89,31 @@ compact_kernel(Shape s, CompactArgs a, const int32_t* __restrict__ cu_kept, cons
 
 namespace {
 
+// Running scores follow the cache: out[l][h][dst] = in[l][h][src] for the kept tokens (or the slots of the kept
+// pages; slots past the end of a sequence get 0).  One thread per (layer, kept row), looping over the heads.
+__global__ void __launch_bounds__(256)
+compact_scores_kernel(Shape s, const float* __restrict__ in, float* __restrict__ out, const int32_t* __restrict__ cu_kept,
+                      const int32_t* __restrict__ idx, long long total_kept, int page_size, long long out_tokens) {
+  const long long out_row = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long row = out_row / page_size;
+  const int slot = (int)(out_row - row * page_size);
+  if (row >= total_kept) return;
+  const int n_seg = s.n_layers * s.n_seqs;
+  int lo = 0, hi = n_seg;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if ((long long)__ldg(cu_kept + mid) <= row) lo = mid; else hi = mid;
+  }
+  const int layer = lo / s.n_seqs, seq = lo - layer * s.n_seqs;
+  const int seq_begin = __ldg(s.cu_seqlens + seq);
+  const long long tok_in_seq = (long long)__ldg(idx + row) * page_size + slot;
+  const bool present = tok_in_seq < __ldg(s.cu_seqlens + seq + 1) - seq_begin;
+  const long long dst = (row - __ldg(cu_kept + layer * s.n_seqs)) * page_size + slot;
+  const float* src = in + (long long)layer * s.Hq * s.T + seq_begin + tok_in_seq;
+  float* dp = out + (long long)layer * s.Hq * out_tokens + dst;
+  for (int h = 0; h < s.Hq; ++h) dp[(long long)h * out_tokens] = present ? __ldg(src + (long long)h * s.T) : 0.f;
+}
+
 int launch_gather(const Shape& s, const TensorView& K, const TensorView* V, int page_size, const int32_t* cu_kept,
                   const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,
                   cudaStream_t stream) {
@@ -122,6 +147,19 @@ int launch_compact(const Shape& s, const TensorView& K, const TensorView* V, con
                    const int32_t* idx, long long total_kept, const TensorView& K_out, const TensorView* V_out,
                    cudaStream_t stream) {
   return launch_gather(s, K, V, 0, cu_kept, idx, total_kept, K_out, V_out, stream);
+}
+
+int launch_compact_scores(const Shape& s, const float* scores_in, int page_size, const int32_t* cu_kept,
+                          const int32_t* idx, long long total_kept, float* scores_out, long long out_tokens,
+                          cudaStream_t stream) {
+  if (total_kept == 0) return KVCRUSH_OK;
+  const int ps = page_size > 0 ? page_size : 1;
+  const long long rows = total_kept * ps;
+  const long long blocks = (rows + 255) / 256;
+  if (blocks > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
+  compact_scores_kernel<<<(unsigned)blocks, 256, 0, stream>>>(s, scores_in, scores_out, cu_kept, idx, total_kept, ps,
+                                                             out_tokens);
+  return check_launch();
 }
 
 int launch_compact_pages(const Shape& s, const TensorView& K, const TensorView* V, int page_size,

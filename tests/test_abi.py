@@ -108,6 +108,10 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
     assert lib.kvcrush_score_decode(r(p), r(t), r(t), None, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_score_decode(r(p), r(t), r(f16), 0x100, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_score_decode(r(p), r(odd), r(t), 0x100, 0x100, None) == B.ERR_MISALIGNED
+    # score gather: aliasing, negative counts
+    assert lib.kvcrush_compact_scores(r(p), 0x100, 0, 0x100, 0x100, 4, 0x100, 16, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_compact_scores(r(p), 0x100, -1, 0x100, 0x100, 4, 0x200, 16, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_compact_scores(r(p), 0x100, 0, 0x100, 0x100, -4, 0x200, 16, 0x100, None) == B.ERR_INVALID_ARG
     # pooling: even kernel, aliasing
     assert lib.kvcrush_pool_scores(r(p), 0x100, 4, 0x200, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_pool_scores(r(p), 0x100, 3, 0x100, 0x100, None) == B.ERR_INVALID_ARG
