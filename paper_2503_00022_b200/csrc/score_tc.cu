@@ -389,7 +389,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (!ok) break;
             tc_fence_after();
             if (g.diag(gi, i))
-              sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
+              sweep_tile<true>(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<true>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
             else
               sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { colsum_piece<false>(v, lse_buf + p * 16, scale2, r, p * 16, acc); }, release);
           }
@@ -416,7 +416,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const int n_valid = g.causal ? (g.diag(gi, i) ? r + 1 : kTile) : min(kTile, g.L - i * kTile);
           // masked columns, or a row that has no reference yet (its first tile): exact maxima, piece by piece
           if (__any_sync(0xFFFFFFFFu, n_valid < kTile || !(m > -3.0e38f)))
-            sweep_tile(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, scale2, n_valid - p * 16, m, sum2); }, release);
+            sweep_tile<true>(t_acc, [&](const uint32_t (&v)[16], int p) { lse_piece<true>(v, scale, scale2, n_valid - p * 16, m, sum2); }, release);
           else
             lse_tile_lazy(t_acc, scale, scale2, m, sum2, release);
         }

@@ -187,20 +187,35 @@ __device__ __forceinline__ void tmem_wait16(uint32_t (&v)[16]) {
 
 // Streams the 128 columns of one accumulator through two 16-column register buffers: the load of the next
 // piece is in flight while the current one is processed.  `release` runs once the last load has landed.
-template <class Piece, class Release>
+// kRolled keeps the loop rolled (two pieces per iteration): for the tile kinds that are rare (diagonal and first
+// tiles), so that their code does not push the common kind out of the instruction cache.
+template <bool kRolled = false, class Piece, class Release>
 __device__ __forceinline__ void sweep_tile(uint32_t taddr, Piece&& piece, Release&& release) {
   uint32_t va[16], vb[16];
   tmem_ld16(taddr, va);
   tmem_wait16(va);
+  if constexpr (kRolled) {
+#pragma unroll 1
+    for (int p = 0; p < 8; p += 2) {
+      tmem_ld16(taddr + (p + 1) * 16, vb);
+      piece(va, p);
+      tmem_wait16(vb);
+      if (p == 6) release();
+      if (p < 6) tmem_ld16(taddr + (p + 2) * 16, va);
+      piece(vb, p + 1);
+      if (p < 6) tmem_wait16(va);
+    }
+  } else {
 #pragma unroll
-  for (int p = 0; p < 8; p += 2) {
-    tmem_ld16(taddr + (p + 1) * 16, vb);
-    piece(va, p);
-    tmem_wait16(vb);
-    if (p == 6) release();
-    if (p < 6) tmem_ld16(taddr + (p + 2) * 16, va);
-    piece(vb, p + 1);
-    if (p < 6) tmem_wait16(va);
+    for (int p = 0; p < 8; p += 2) {
+      tmem_ld16(taddr + (p + 1) * 16, vb);
+      piece(va, p);
+      tmem_wait16(vb);
+      if (p == 6) release();
+      if (p < 6) tmem_ld16(taddr + (p + 2) * 16, va);
+      piece(vb, p + 1);
+      if (p < 6) tmem_wait16(va);
+    }
   }
 }
 
