@@ -34,7 +34,7 @@ from paper_2503_00022_b200 import inputs  # noqa: E402
 METRIC = "prompt tokens compressed/s (score+select+compact)"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg3_llama2_32l_8k"
-NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP = 138.4e6   # (275.5 + 278.2) MB / 2 sweeps / 2 layers: dram__bytes_read + dram__bytes_write
+NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP = 138.2e6   # (276.0 + 276.7) MB / 2 sweeps / 2 layers: dram__bytes_read + dram__bytes_write
 
 
 def measured_peaks():
