@@ -16,7 +16,9 @@
  *   - Pointers named *_dev (and every tensor / output pointer) are DEVICE pointers
  *     owned by the caller; pointers named *_host are host pointers read during the
  *     call only.  The library allocates and frees no memory and keeps no state
- *     between calls; scratch memory is the caller's `workspace` (device, 256-byte
+ *     between calls apart from two process-wide, write-once caches (the driver's
+ *     tensor-map encoder entry point; for kvcrush_signature_static the device address
+ *     of its array); scratch memory is the caller's `workspace` (device, 256-byte
  *     aligned, size from kvcrush_workspace_size).
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
  *     stream) and the call returns without synchronising.  Inputs are never written.
@@ -74,7 +76,8 @@ extern "C" {
 #define KVCRUSH_ANCHOR_EXPLICIT  2   /* caller's bits (a seeded random anchor is drawn on the host) */
 
 /* score kernels */
-#define KVCRUSH_SCORE_AUTO       0   /* tensor-core kernels when the shape allows, else SIMT  */
+#define KVCRUSH_SCORE_AUTO       0   /* tensor-core kernels when type, shape and strides allow, else SIMT;
+                                        never a silent drop to SIMT because the driver lacks something  */
 #define KVCRUSH_SCORE_SIMT       1   /* fp32 CUDA-core kernels (any supported shape and type) */
 #define KVCRUSH_SCORE_TENSOR     2   /* tcgen05 kernels, error if the shape is not supported  */
 
@@ -129,9 +132,15 @@ int kvcrush_workspace_size(const kvcrush_problem_t* problem, int stage, size_t* 
  *   scores_dev  out [n_layers][n_q_heads][T] float32
  *   lse_out_dev optional out, same shape: the row log-sum-exp (natural log);
  *               not written when lse_in_dev is given
- *   impl        KVCRUSH_SCORE_*
- *   workspace   kvcrush_workspace_size(.., KVCRUSH_STAGE_SCORE, ..) bytes (always required: it also
- *               holds the kernels' work counters)
+ *   impl        KVCRUSH_SCORE_AUTO takes the tensor-core kernels when Q and K are BF16 or FP16, head_dim is a
+ *               multiple of 8 up to 128 and the strides can be described to the TMA unit (a stride of 0 along an
+ *               axis longer than 1, or beyond the tensor map's limits, cannot), otherwise the CUDA-core kernels.
+ *               When the problem qualifies but the driver does not provide the tensor-map encoder, AUTO returns
+ *               KVCRUSH_ERR_UNSUPPORTED rather than running the (about 100 times slower) CUDA-core kernels
+ *               unnoticed; ask for KVCRUSH_SCORE_SIMT explicitly in that case.  KVCRUSH_SCORE_TENSOR returns
+ *               KVCRUSH_ERR_UNSUPPORTED for anything the tensor-core kernels cannot take.
+ *   workspace   kvcrush_workspace_size(.., KVCRUSH_STAGE_SCORE, ..) bytes; with lse_in_dev given only the first
+ *               256 bytes are used (the kernels' work counters) and a 256-byte workspace is enough
  */
 int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, const kvcrush_tensor_t* K,
                   const float* lse_in_dev, float* scores_dev, float* lse_out_dev, int normalize, int impl,
@@ -149,7 +158,8 @@ int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, c
  *   Q_new       [n_layers][n_seqs][n_q_heads][head_dim]: stride_token steps from one sequence to the next
  *   K           the cached keys, token-major, same dtype as Q_new (BF16, FP16 or FP32), head_dim <= 256, multiple of 8
  *   scores_dev  in/out [n_layers][n_q_heads][T] float32 running column sums
- * Runs on the CUDA cores (one block per layer, sequence and query head); bound by reading K twice.
+ * Runs on the CUDA cores (one block per layer, sequence and KV head, which serves the query heads of its group);
+ * bound by reading K twice.
  */
 int kvcrush_score_decode(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q_new, const kvcrush_tensor_t* K,
                          float* scores_dev, int32_t* status_dev, void* stream);
@@ -165,10 +175,14 @@ int kvcrush_score_decode(const kvcrush_problem_t* problem, const kvcrush_tensor_
  *                  (the input form of Algorithm 1)
  *   sigs_dev       out [n_layers][T][W] uint32
  *   theta_out_dev  optional out [n_layers][n_seqs][n_q_heads] float32
+ *   importance_out_dev  optional out [n_layers][T] float64: the token importance I(t) that stage 3 ranks (the
+ *                  sum of the token's per-head scores in the order kvcrush_select states), written from the
+ *                  loads this stage does anyway; hand it to kvcrush_select / kvcrush_select_pages as
+ *                  importance_dev and they skip their own pass over the scores
  *   workspace      holds the thresholds when theta_out_dev is NULL
  */
 int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev, const int32_t* sig_keep_dev,
-                      const float* theta_in_dev, uint32_t* sigs_dev, float* theta_out_dev,
+                      const float* theta_in_dev, uint32_t* sigs_dev, float* theta_out_dev, double* importance_out_dev,
                       void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
 /*
@@ -182,6 +196,9 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
  *   rep_i = member of bucket i closest to the bucket's per-bit mean (L1; ties: lower t)
  *   kept  = Imp U {rep_i}, ascending token index.  budget_imp + budget_rep >= length
  *           keeps every token.
+ *   scores_dev         [n_layers][n_q_heads][T] float32; may be NULL when importance_dev is given
+ *   importance_dev     optional [n_layers][T] float64: I(t) as kvcrush_signature writes it (importance_out_dev);
+ *                      NULL: computed here from scores_dev
  *   budget_imp_dev, budget_rep_dev  [n_layers][n_seqs] int32, >= 0
  *   anchor_mode        KVCRUSH_ANCHOR_*
  *   anchor_bits_dev    [W] uint32 (anchor_per_segment == 0) or [n_layers][n_seqs][W];
@@ -195,13 +212,15 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
  *                      prefix sums of min(budget_imp + budget_rep, length)
  *   idx_dev            out [cu_kept[last]] int32 token index inside its sequence
  *   kind_dev           optional out, same length, uint8: 0 important, 1 representative
+ *   n_kept_dev         optional out [n_layers][n_seqs] int32: tokens kept of every segment,
+ *                      min(budget_imp + budget_rep, length) - what cu_kept's differences must be
  * Sequences longer than 262144 tokens are not supported.
  */
-int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
-                   const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const double* importance_dev,
+                   const uint32_t* sigs_dev, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
                    int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
                    int keep_initial, int keep_recent,
-                   const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev,
+                   const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev, int32_t* n_kept_dev,
                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
 /*
@@ -241,6 +260,8 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
  *   then exactly the steps of kvcrush_select on the other pages: d_p = popcount(v_p xor anchor), (d_p, p) order,
  *   budget_rep equal-frequency buckets, per bucket the page closest to the per-bit mean (L1; ties: lower page),
  *   kept = Imp U representatives, ascending.  budget_imp + budget_rep >= number of pages keeps every page.
+ *   scores_dev,        as for kvcrush_select: the token importance comes from importance_dev when given, else from
+ *   importance_dev     the scores
  *   page_size          >= 1; page_size * W <= 128 words and at most 8192 pages per sequence, otherwise
  *                      KVCRUSH_ERR_UNSUPPORTED.  page_size 1 gives the result of kvcrush_select.
  *   anchor_bits_dev    [W] or [n_layers][n_seqs][W] token anchor (EXPLICIT only)
@@ -249,13 +270,15 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
  *   cu_kept_dev        [n_layers*n_seqs + 1] prefix sums of min(budget_imp + budget_rep, pages of the sequence)
  *   page_idx_dev       out [cu_kept[last]] int32 page number inside its sequence
  *   kind_dev           optional out: 0 important, 1 representative
+ *   n_kept_dev         optional out [n_layers][n_seqs] int32: pages kept of every segment
  *   workspace          kvcrush_workspace_size(.., KVCRUSH_STAGE_SELECT, ..) bytes
  */
-int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
-                         int page_size, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_dev, const double* importance_dev,
+                         const uint32_t* sigs_dev, int page_size,
+                         const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
                          int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
                          int keep_initial, int keep_recent,
-                         const int32_t* cu_kept_dev, int32_t* page_idx_dev, uint8_t* kind_dev,
+                         const int32_t* cu_kept_dev, int32_t* page_idx_dev, uint8_t* kind_dev, int32_t* n_kept_dev,
                          void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
 /*

@@ -71,11 +71,11 @@ def lib() -> ctypes.CDLL:
         L.kvcrush_score.argtypes = [P, T, T, vp, vp, vp, i32, i32, vp, sz, vp, vp]
         L.kvcrush_score_decode.argtypes = [P, T, T, vp, vp, vp]
         L.kvcrush_compact_scores.argtypes = [P, vp, i32, vp, vp, i64, vp, i64, vp, vp]
-        L.kvcrush_signature.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp]
-        L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
+        L.kvcrush_signature.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_pool_scores.argtypes = [P, vp, i32, vp, vp, vp]
         L.kvcrush_compact.argtypes = [P, T, T, vp, vp, i64, T, T, vp, vp]
-        L.kvcrush_select_pages.argtypes = [P, vp, vp, i32, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
+        L.kvcrush_select_pages.argtypes = [P, vp, vp, vp, i32, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_compact_pages.argtypes = [P, T, T, i32, vp, vp, i64, T, T, vp, vp]
         L.kvcrush_signature_static.argtypes = [P, vp, vp, vp, vp, vp]
         L.kvcrush_strerror.argtypes = [i32]
@@ -179,10 +179,10 @@ def kvcrush_compact_scores(problem: Problem, scores_in, page_size: int, cu_kept,
 
 
 def kvcrush_signature(problem: Problem, scores, sigs, *, sig_keep=None, theta_in=None, theta_out=None,
-                      workspace=None, status=None, stream: Optional[int] = None) -> None:
+                      importance_out=None, workspace=None, status=None, stream: Optional[int] = None) -> None:
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().kvcrush_signature(problem.ref, _ptr(scores), _ptr(sig_keep), _ptr(theta_in), _ptr(sigs),
-                                   _ptr(theta_out), _ptr(workspace), ws_bytes, _ptr(status),
+                                   _ptr(theta_out), _ptr(importance_out), _ptr(workspace), ws_bytes, _ptr(status),
                                    _stream() if stream is None else stream), "kvcrush_signature")
 
 
@@ -195,14 +195,14 @@ def kvcrush_signature_static(problem: Problem, scores, sigs, sig_keep, *, status
                                           _stream() if stream is None else stream), "kvcrush_signature_static")
 
 
-def kvcrush_select(problem: Problem, scores, sigs, budget_imp, budget_rep, cu_kept, idx, *, kind=None,
-                   anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None, anchor_per_segment=False, keep_recent=0,
+def kvcrush_select(problem: Problem, scores, sigs, budget_imp, budget_rep, cu_kept, idx, *, importance=None,
+                   kind=None, n_kept=None, anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None, anchor_per_segment=False, keep_recent=0,
                    keep_initial=0, workspace=None, status=None, stream: Optional[int] = None) -> None:
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    _check(lib().kvcrush_select(problem.ref, _ptr(scores), _ptr(sigs), _ptr(budget_imp), _ptr(budget_rep),
+    _check(lib().kvcrush_select(problem.ref, _ptr(scores), _ptr(importance), _ptr(sigs), _ptr(budget_imp), _ptr(budget_rep),
                                 int(anchor_mode), _ptr(anchor_bits), int(anchor_per_segment), int(keep_initial),
                                 int(keep_recent), _ptr(cu_kept),
-                                _ptr(idx), _ptr(kind), _ptr(workspace), ws_bytes, _ptr(status),
+                                _ptr(idx), _ptr(kind), _ptr(n_kept), _ptr(workspace), ws_bytes, _ptr(status),
                                 _stream() if stream is None else stream), "kvcrush_select")
 
 
@@ -224,13 +224,15 @@ def kvcrush_compact(problem: Problem, k, v, cu_kept, idx, total_kept: int, k_out
 
 
 def kvcrush_select_pages(problem: Problem, scores, sigs, page_size: int, budget_imp, budget_rep, cu_kept, page_idx, *,
-                         kind=None, anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None, anchor_per_segment=False,
+                         importance=None, kind=None, n_kept=None, anchor_mode=ANCHOR_ALTERNATE, anchor_bits=None,
+                         anchor_per_segment=False,
                          keep_initial=0, keep_recent=0, workspace=None, status=None,
                          stream: Optional[int] = None) -> None:
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    _check(lib().kvcrush_select_pages(problem.ref, _ptr(scores), _ptr(sigs), int(page_size), _ptr(budget_imp),
+    _check(lib().kvcrush_select_pages(problem.ref, _ptr(scores), _ptr(importance), _ptr(sigs), int(page_size), _ptr(budget_imp),
                                       _ptr(budget_rep), int(anchor_mode), _ptr(anchor_bits), int(anchor_per_segment),
-                                      int(keep_initial), int(keep_recent), _ptr(cu_kept), _ptr(page_idx), _ptr(kind), _ptr(workspace), ws_bytes,
+                                      int(keep_initial), int(keep_recent), _ptr(cu_kept), _ptr(page_idx), _ptr(kind), _ptr(n_kept),
+                                      _ptr(workspace), ws_bytes,
                                       _ptr(status), _stream() if stream is None else stream), "kvcrush_select_pages")
 
 
@@ -260,7 +262,8 @@ class CompressionPass:
     def __init__(self, problem: Problem, budget_imp: np.ndarray, budget_rep: np.ndarray,
                  cache_dtype=None, sig_keep: Optional[np.ndarray] = None, anchor_mode=ANCHOR_ALTERNATE,
                  anchor_bits: Optional[np.ndarray] = None, impl=SCORE_AUTO, with_kind=True, with_cache=True,
-                 pool_kernel: int = 0, keep_recent: int = 0, page_size: int = 0, keep_initial: int = 0):
+                 pool_kernel: int = 0, keep_recent: int = 0, page_size: int = 0, keep_initial: int = 0,
+                 share_importance: bool = True):
         import torch
         self.page_size = int(page_size)
         unit = max(self.page_size, 1)
@@ -295,6 +298,10 @@ class CompressionPass:
         self.sigs = torch.empty((Lyr, T, p.W), dtype=torch.int32, device=dev)
         self.idx = torch.empty((max(self.total_kept, 1),), dtype=torch.int32, device=dev)
         self.kind = torch.empty((max(self.total_kept, 1),), dtype=torch.uint8, device=dev) if with_kind else None
+        self.n_kept = torch.empty((Lyr, S), dtype=torch.int32, device=dev)
+        # token importance handed from the signature stage to the selection stage (one pass over the scores saved)
+        self.importance = torch.empty((Lyr, T), dtype=torch.float64, device=dev) if share_importance else None
+        self._importance_of = None          # data pointer of the scores the importance was computed from
         self.status = torch.zeros(4, dtype=torch.int32, device=dev)
         nbytes = max(kvcrush_workspace_size(p, st) for st in (STAGE_SCORE, STAGE_SIGNATURE, STAGE_SELECT))
         self.workspace = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=dev)
@@ -319,19 +326,25 @@ class CompressionPass:
         return self.pooled if self.pooled is not None else self.scores
 
     def signature(self, scores=None):
-        kvcrush_signature(self.problem, self._selection_scores(scores), self.sigs,
-                          sig_keep=self.sig_keep, theta_out=self.theta, workspace=self.workspace, status=self.status)
+        sc = self._selection_scores(scores)
+        kvcrush_signature(self.problem, sc, self.sigs, sig_keep=self.sig_keep, theta_out=self.theta,
+                          importance_out=self.importance, workspace=self.workspace, status=self.status)
+        self._importance_of = None if self.importance is None else int(sc.data_ptr())
 
     def select(self, scores=None):
+        sc = self._selection_scores(scores)
+        imp = self.importance if self._importance_of == int(sc.data_ptr()) else None
         if self.page_size:
-            kvcrush_select_pages(self.problem, self._selection_scores(scores), self.sigs, self.page_size,
-                                 self.budget_imp, self.budget_rep, self.cu_kept, self.idx, kind=self.kind,
-                                 anchor_mode=self.anchor_mode, anchor_bits=self.anchor_bits,
+            kvcrush_select_pages(self.problem, sc, self.sigs, self.page_size, importance=imp,
+                                 budget_imp=self.budget_imp, budget_rep=self.budget_rep, cu_kept=self.cu_kept,
+                                 page_idx=self.idx, kind=self.kind,
+                                 n_kept=self.n_kept, anchor_mode=self.anchor_mode, anchor_bits=self.anchor_bits,
                                  keep_initial=self.keep_initial, keep_recent=self.keep_recent,
                                  workspace=self.workspace, status=self.status)
             return
-        kvcrush_select(self.problem, self._selection_scores(scores), self.sigs, self.budget_imp,
-                       self.budget_rep, self.cu_kept, self.idx, kind=self.kind, anchor_mode=self.anchor_mode,
+        kvcrush_select(self.problem, sc, self.sigs, self.budget_imp,
+                       self.budget_rep, self.cu_kept, self.idx, importance=imp, kind=self.kind, n_kept=self.n_kept,
+                       anchor_mode=self.anchor_mode,
                        anchor_bits=self.anchor_bits, keep_recent=self.keep_recent, keep_initial=self.keep_initial,
                        workspace=self.workspace, status=self.status)
 

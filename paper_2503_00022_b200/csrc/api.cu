@@ -48,8 +48,9 @@ int make_view(const kvcrush_tensor_t* t, int head_dim, TensorView* v) {
 }
 
 size_t score_lse_bytes(const Shape& s) { return round_up((size_t)s.n_layers * s.Hq * s.T * sizeof(float)); }
-// row log-sum-exp of every query + the work counters of the persistent tensor-core kernels
-size_t score_ws(const Shape& s) { return score_lse_bytes(s) + round_up(score_tensor_counter_bytes()); }
+// work counters of the persistent tensor-core kernels first, then the row log-sum-exp of every query
+size_t score_counter_bytes() { return round_up(score_tensor_counter_bytes()); }
+size_t score_ws(const Shape& s) { return score_counter_bytes() + score_lse_bytes(s); }
 size_t signature_ws(const Shape& s) { return round_up((size_t)s.n_layers * s.n_seqs * s.Hq * sizeof(float)); }
 
 }  // namespace
@@ -74,9 +75,13 @@ int kvcrush_workspace_size(const kvcrush_problem_t* problem, int stage, size_t* 
   }
 }
 
-int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, const kvcrush_tensor_t* K,
-                  const float* lse_in_dev, float* scores_dev, float* lse_out_dev, int normalize, int impl,
-                  void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+}  // extern "C"
+
+namespace {
+
+int score_entry(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, const kvcrush_tensor_t* K,
+                const float* lse_in_dev, float* scores_dev, float* lse_out_dev, int normalize, int impl,
+                void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream, const ScoreDiag& diag) {
   Shape s;
   int rc = make_shape(problem, &s);
   if (rc != KVCRUSH_OK) return rc;
@@ -87,21 +92,54 @@ int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, c
   if (q.dtype != k.dtype) return KVCRUSH_ERR_INVALID_ARG;
   if (impl != KVCRUSH_SCORE_AUTO && impl != KVCRUSH_SCORE_SIMT && impl != KVCRUSH_SCORE_TENSOR)
     return KVCRUSH_ERR_INVALID_ARG;
-  if (!workspace || workspace_bytes < score_ws(s)) return KVCRUSH_ERR_WORKSPACE;
+  // with the row log-sum-exp supplied only the work counters live in the workspace
+  if (!workspace || workspace_bytes < (lse_in_dev ? score_counter_bytes() : score_ws(s))) return KVCRUSH_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
-  float* lse2_ws = static_cast<float*>(workspace);
-  int* counters = reinterpret_cast<int*>(static_cast<unsigned char*>(workspace) + score_lse_bytes(s));
+  int* counters = static_cast<int*>(workspace);
+  float* lse2_ws = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + score_counter_bytes());
   const float scale = problem->softmax_scale != 0.f ? problem->softmax_scale : 1.f / sqrtf((float)s.D);
   const float log2e = 1.4426950408889634f;
   const float scale_log2 = scale * log2e;
-  const bool tensor_ok = score_tensor_supported(s, q, k);
-  if (impl == KVCRUSH_SCORE_TENSOR && !tensor_ok) return KVCRUSH_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (impl == KVCRUSH_SCORE_SIMT || !tensor_ok)
+  ScoreTensorMaps maps;
+  const int plan = impl == KVCRUSH_SCORE_SIMT ? TENSOR_PLAN_NO : score_tensor_plan(s, q, k, &maps);
+  // a problem made for the tensor cores must not end up on the CUDA cores because the driver lacks the encoder
+  if (plan == TENSOR_PLAN_NO_ENCODER) return KVCRUSH_ERR_UNSUPPORTED;
+  if (plan == TENSOR_PLAN_NO) {
+    if (impl == KVCRUSH_SCORE_TENSOR) return KVCRUSH_ERR_UNSUPPORTED;
     return launch_score_simt(s, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, scores_dev, lse_out_dev, normalize,
                              status_dev, st);
-  return launch_score_tensor(s, problem->cu_seqlens_host, q, k, scale_log2, lse_in_dev, log2e, lse2_ws, counters,
-                             scores_dev, lse_out_dev, normalize, status_dev, st);
+  }
+  return launch_score_tensor(s, problem->cu_seqlens_host, q, maps, scale_log2, lse_in_dev, log2e, lse2_ws, counters,
+                             scores_dev, lse_out_dev, normalize, status_dev, diag, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int kvcrush_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, const kvcrush_tensor_t* K,
+                  const float* lse_in_dev, float* scores_dev, float* lse_out_dev, int normalize, int impl,
+                  void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  return score_entry(problem, Q, K, lse_in_dev, scores_dev, lse_out_dev, normalize, impl, workspace, workspace_bytes,
+                     status_dev, stream, ScoreDiag{});
+}
+
+// Not part of the public ABI (the header does not declare it): kvcrush_score with the diagnostics of the tensor-core
+// kernels exposed, for the test that makes a bounded wait run out.  short_waits != 0 runs the instantiation of the
+// kernels whose barrier waits give up after a few thousand polls; withhold_first_item != 0 makes the producer warp of
+// every CTA stop after fetching its first work item, before announcing it and before issuing any copy, so that the
+// other roles' first waits run out with nothing in flight: the kernels return normally with
+// status = {KVCRUSH_DEV_TIMEOUT, kernel id, block, 0}.
+int kvcrush_diag_score(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q, const kvcrush_tensor_t* K,
+                       const float* lse_in_dev, float* scores_dev, float* lse_out_dev, int normalize, int impl,
+                       void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream,
+                       int short_waits, int withhold_first_item) {
+  ScoreDiag diag{};
+  diag.short_waits = short_waits != 0;
+  diag.withhold_first_item = withhold_first_item != 0;
+  return score_entry(problem, Q, K, lse_in_dev, scores_dev, lse_out_dev, normalize, impl, workspace, workspace_bytes,
+                     status_dev, stream, diag);
 }
 
 int kvcrush_score_decode(const kvcrush_problem_t* problem, const kvcrush_tensor_t* Q_new, const kvcrush_tensor_t* K,
@@ -119,7 +157,7 @@ int kvcrush_score_decode(const kvcrush_problem_t* problem, const kvcrush_tensor_
 }
 
 int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev, const int32_t* sig_keep_dev,
-                      const float* theta_in_dev, uint32_t* sigs_dev, float* theta_out_dev,
+                      const float* theta_in_dev, uint32_t* sigs_dev, float* theta_out_dev, double* importance_out_dev,
                       void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
   Shape s;
   const int rc = make_shape(problem, &s);
@@ -137,20 +175,23 @@ int kvcrush_signature(const kvcrush_problem_t* problem, const float* scores_dev,
                         cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return KVCRUSH_ERR_CUDA;
   }
-  return launch_signature(s, scores_dev, sig_keep_dev, theta_in_dev, sigs_dev, theta, st);
+  if (importance_out_dev && reinterpret_cast<uintptr_t>(importance_out_dev) % 8) return KVCRUSH_ERR_MISALIGNED;
+  return launch_signature(s, scores_dev, sig_keep_dev, theta_in_dev, sigs_dev, theta, importance_out_dev, st);
 }
 
-int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
-                   const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, const double* importance_dev,
+                   const uint32_t* sigs_dev, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
                    int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
                    int keep_initial, int keep_recent,
-                   const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev,
+                   const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev, int32_t* n_kept_dev,
                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
   Shape s;
   const int rc = make_shape(problem, &s);
   if (rc != KVCRUSH_OK) return rc;
-  if (!scores_dev || !sigs_dev || !budget_imp_dev || !budget_rep_dev || !cu_kept_dev || !idx_dev || !status_dev)
+  if ((!scores_dev && !importance_dev) || !sigs_dev || !budget_imp_dev || !budget_rep_dev || !cu_kept_dev || !idx_dev ||
+      !status_dev)
     return KVCRUSH_ERR_INVALID_ARG;
+  if (importance_dev && reinterpret_cast<uintptr_t>(importance_dev) % 8) return KVCRUSH_ERR_MISALIGNED;
   if (anchor_mode != KVCRUSH_ANCHOR_ALTERNATE && anchor_mode != KVCRUSH_ANCHOR_MEAN &&
       anchor_mode != KVCRUSH_ANCHOR_EXPLICIT)
     return KVCRUSH_ERR_INVALID_ARG;
@@ -159,9 +200,9 @@ int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, co
   if (s.max_seqlen > 262144) return KVCRUSH_ERR_UNSUPPORTED;
   if (!workspace || workspace_bytes < select_workspace_bytes(s)) return KVCRUSH_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
-  return launch_select(s, scores_dev, sigs_dev, budget_imp_dev, budget_rep_dev, anchor_mode, anchor_bits_dev,
-                       anchor_per_segment != 0, keep_initial, keep_recent, cu_kept_dev, idx_dev, kind_dev, workspace,
-                       static_cast<cudaStream_t>(stream));
+  return launch_select(s, scores_dev, importance_dev, sigs_dev, budget_imp_dev, budget_rep_dev, anchor_mode, anchor_bits_dev,
+                       anchor_per_segment != 0, keep_initial, keep_recent, cu_kept_dev, idx_dev, kind_dev, n_kept_dev,
+                       workspace, static_cast<cudaStream_t>(stream));
 }
 
 int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K, const kvcrush_tensor_t* V,
@@ -186,17 +227,19 @@ int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K,
                         static_cast<cudaStream_t>(stream));
 }
 
-int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_dev, const uint32_t* sigs_dev,
-                         int page_size, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_dev, const double* importance_dev,
+                         const uint32_t* sigs_dev, int page_size, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
                          int anchor_mode, const uint32_t* anchor_bits_dev, int anchor_per_segment,
                          int keep_initial, int keep_recent,
-                         const int32_t* cu_kept_dev, int32_t* page_idx_dev, uint8_t* kind_dev,
+                         const int32_t* cu_kept_dev, int32_t* page_idx_dev, uint8_t* kind_dev, int32_t* n_kept_dev,
                          void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
   Shape s;
   const int rc = make_shape(problem, &s);
   if (rc != KVCRUSH_OK) return rc;
-  if (!scores_dev || !sigs_dev || !budget_imp_dev || !budget_rep_dev || !cu_kept_dev || !page_idx_dev || !status_dev)
+  if ((!scores_dev && !importance_dev) || !sigs_dev || !budget_imp_dev || !budget_rep_dev || !cu_kept_dev ||
+      !page_idx_dev || !status_dev)
     return KVCRUSH_ERR_INVALID_ARG;
+  if (importance_dev && reinterpret_cast<uintptr_t>(importance_dev) % 8) return KVCRUSH_ERR_MISALIGNED;
   if (anchor_mode != KVCRUSH_ANCHOR_ALTERNATE && anchor_mode != KVCRUSH_ANCHOR_MEAN &&
       anchor_mode != KVCRUSH_ANCHOR_EXPLICIT)
     return KVCRUSH_ERR_INVALID_ARG;
@@ -206,9 +249,9 @@ int kvcrush_select_pages(const kvcrush_problem_t* problem, const float* scores_d
   if (((long long)s.max_seqlen + page_size - 1) / page_size > kMaxPagesPerSeq) return KVCRUSH_ERR_UNSUPPORTED;
   if (!workspace || workspace_bytes < select_workspace_bytes(s)) return KVCRUSH_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
-  return launch_select_pages(s, scores_dev, sigs_dev, page_size, budget_imp_dev, budget_rep_dev, anchor_mode,
+  return launch_select_pages(s, scores_dev, importance_dev, sigs_dev, page_size, budget_imp_dev, budget_rep_dev, anchor_mode,
                              anchor_bits_dev, anchor_per_segment != 0, keep_initial, keep_recent, cu_kept_dev,
-                             page_idx_dev, kind_dev,
+                             page_idx_dev, kind_dev, n_kept_dev,
                              workspace, static_cast<cudaStream_t>(stream));
 }
 

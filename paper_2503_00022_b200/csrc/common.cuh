@@ -56,21 +56,35 @@ int launch_score_simt(const Shape& s, const TensorView& Q, const TensorView& K, 
 // Decode step: scores[l][h][t] += attention of sequence(t)'s new query (Q_new's token axis = sequence) to key t.
 int launch_score_decode(const Shape& s, const TensorView& Q_new, const TensorView& K, float scale_log2, float* scores,
                         cudaStream_t stream);
-bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorView& K);
+// Can the tensor-core kernels take this problem?  On TENSOR_PLAN_OK `maps` holds the two encoded tensor maps.
+enum { TENSOR_PLAN_OK = 0,
+       TENSOR_PLAN_NO = 1,            // type, head_dim or strides outside what the kernels / the TMA unit take
+       TENSOR_PLAN_NO_ENCODER = 2 };  // the problem qualifies but the driver has no tensor-map encoder
+struct ScoreTensorMaps { alignas(64) unsigned char q[128]; alignas(64) unsigned char k[128]; };   // two CUtensorMap
+int score_tensor_plan(const Shape& s, const TensorView& Q, const TensorView& K, ScoreTensorMaps* maps);
+// Diagnostics of one launch (all zero in normal use).
+struct ScoreDiag {
+  int short_waits;           // run the kernels instantiated with a short limit on every bounded barrier wait
+  int withhold_first_item;   // the producer warp of every CTA stops before announcing its first work item
+};
 // `counters`: two ints of caller scratch (work counters of the two persistent sweeps).
 size_t score_tensor_counter_bytes();
-int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView& Q, const TensorView& K,
+int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView& Q, const ScoreTensorMaps& maps,
                         float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws, int* counters,
-                        float* scores, float* lse_out, int normalize, int32_t* status, cudaStream_t stream);
+                        float* scores, float* lse_out, int normalize, int32_t* status, const ScoreDiag& diag,
+                        cudaStream_t stream);
 
+// importance: optional out [n_layers][T] float64, the token importance I(t) of stage 3 (written from the same loads).
 int launch_signature(const Shape& s, const float* scores, const int32_t* sig_keep, const float* theta_in,
-                     uint32_t* sigs, float* theta, cudaStream_t stream);
+                     uint32_t* sigs, float* theta, double* importance, cudaStream_t stream);
 
 size_t select_workspace_bytes(const Shape& s);
-int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, const int32_t* budget_imp,
+// importance: optional [n_layers][T] float64 I(t) from the signature stage; NULL: computed from the scores.
+int launch_select(const Shape& s, const float* scores, const double* importance, const uint32_t* sigs,
+                  const int32_t* budget_imp,
                   const int32_t* budget_rep, int anchor_mode, const uint32_t* anchor_bits, int anchor_per_segment,
-                  int keep_initial, int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws,
-                  cudaStream_t stream);
+                  int keep_initial, int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind,
+                  int32_t* n_kept, void* ws, cudaStream_t stream);
 
 // Order-preserving 64-bit keys of the token importance I(t), [n_layers][T] (first kernel of the selection stages).
 int launch_importance(const Shape& s, const float* scores, int keep_initial, int keep_recent,
@@ -79,10 +93,12 @@ int launch_importance(const Shape& s, const float* scores, int keep_initial, int
 // Page-granular selection and gather (a page = page_size consecutive tokens of one sequence).
 constexpr int kMaxPagesPerSeq = 8192;      // pages of one sequence the page kernel holds in shared memory
 constexpr int kMaxPageWords = 128;         // signature words of one page (page_size * W)
-int launch_select_pages(const Shape& s, const float* scores, const uint32_t* sigs, int page_size,
+int launch_select_pages(const Shape& s, const float* scores, const double* importance, const uint32_t* sigs,
+                        int page_size,
                         const int32_t* budget_imp, const int32_t* budget_rep, int anchor_mode,
                         const uint32_t* anchor_bits, int anchor_per_segment, int keep_initial, int keep_recent,
-                        const int32_t* cu_kept, int32_t* page_idx, uint8_t* kind, void* ws, cudaStream_t stream);
+                        const int32_t* cu_kept, int32_t* page_idx, uint8_t* kind, int32_t* n_kept, void* ws,
+                        cudaStream_t stream);
 int launch_compact_pages(const Shape& s, const TensorView& K, const TensorView* V, int page_size,
                          const int32_t* cu_kept, const int32_t* page_idx, long long total_kept_pages,
                          const TensorView& K_out, const TensorView* V_out, cudaStream_t stream);

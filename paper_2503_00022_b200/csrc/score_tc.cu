@@ -70,6 +70,8 @@ struct PersistArgs {
   int total_items;         // n_items * n_layers * Hq
   int* counter;            // work counter, zero at launch
   int32_t* status;
+  int withhold_first_item; // diagnostic: the producer warp fetches its first item and then stops before announcing
+                           // it or issuing any copy for it, so that every consumer's first wait runs out
 };
 
 template <int D>
@@ -144,7 +146,8 @@ struct Geo {
   }
 };
 
-template <int D, bool kColsum>
+// kPolls: polls of every bounded barrier wait (a compile-time constant: the epilogue has no register to spare for it).
+template <int D, bool kColsum, uint32_t kPolls>
 __global__ void __launch_bounds__(kThreads, 1)
 score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const PersistArgs a) {
@@ -203,7 +206,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       int idx = 0;
       bool ok = true;
       if (lane == 0) {
-        ok = mbar_wait(smem_u32(&aux->item_empty[slot]), ((n_item >> 1) & 1) ^ 1, abort_flag);
+        ok = mbar_wait(smem_u32(&aux->item_empty[slot]), ((n_item >> 1) & 1) ^ 1, abort_flag, kPolls);
         if (ok) idx = atomicAdd(a.counter, 1);
       }
       ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
@@ -213,6 +216,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (lane == 0) { aux->item[slot][0] = -1; mbar_arrive(smem_u32(&aux->item_full[slot])); }
         break;
       }
+      if (a.withhold_first_item) break;        // nothing is in flight: the consumers' bounded waits end the CTA
       const int lh = idx / a.n_items, rank = idx - lh * a.n_items;
       int seq, blk, nblk;
       decode_item(s.cu_seqlens, s.n_seqs, a.max_blocks, rank, !kColsum, lane, seq, blk, nblk, kBlockRows, s.window);
@@ -224,7 +228,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const Geo<kColsum> g(s, it);
         const int head_fixed = kColsum ? g.hk : g.h, head_stream = kColsum ? g.h : g.hk;
         // the stationary buffer is free once every MMA of the previous item has retired
-        ok = mbar_wait(smem_u32(&aux->fixed_empty), (n_item & 1) ^ 1, abort_flag);
+        ok = mbar_wait(smem_u32(&aux->fixed_empty), (n_item & 1) ^ 1, abort_flag, kPolls);
         if (ok) {
           const int n_slots = g.n_slots();
           mbar_expect_tx(smem_u32(&aux->fixed_full), n_slots * SL::kTileBytes);
@@ -236,7 +240,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           issued_item = n_item + 1;
           for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
             const int rs = n_stream % kRing;
-            ok = mbar_wait(smem_u32(&aux->empty[rs]), ((n_stream / kRing) & 1) ^ 1, abort_flag);
+            ok = mbar_wait(smem_u32(&aux->empty[rs]), ((n_stream / kRing) & 1) ^ 1, abort_flag, kPolls);
             if (!ok) break;
             mbar_expect_tx(smem_u32(&aux->full[rs]), SL::kTileBytes);
 #pragma unroll
@@ -253,9 +257,9 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (lane == 0 && *abort_flag) {
       // give the copies in flight a bounded time to land before the CTA's shared memory is released
       for (int q = max(0, n_stream - kRing); q < n_stream; ++q)
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->full[q % kRing]), (q / kRing) & 1); ++i) {}
+        for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(smem_u32(&aux->full[q % kRing]), (q / kRing) & 1); ++i) {}
       if (issued_item > 0)
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->fixed_full), (issued_item - 1) & 1); ++i) {}
+        for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(smem_u32(&aux->fixed_full), (issued_item - 1) & 1); ++i) {}
     }
   } else if (warp <= kIssueWarps) {
     // ------------------------------ MMA issuers ------------------------------
@@ -269,7 +273,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       bool ok = true;
       while (ok) {
         const int slot = n_item & 1;
-        ok = mbar_wait(smem_u32(&aux->item_full[slot]), (n_item >> 1) & 1, abort_flag);
+        ok = mbar_wait(smem_u32(&aux->item_full[slot]), (n_item >> 1) & 1, abort_flag, kPolls);
         if (!ok) break;
         int it[5];
 #pragma unroll
@@ -277,12 +281,12 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         mbar_arrive(smem_u32(&aux->item_empty[slot]));
         if (it[0] < 0) break;
         const Geo<kColsum> g(s, it);
-        ok = mbar_wait(smem_u32(&aux->fixed_full), n_item & 1, abort_flag);
+        ok = mbar_wait(smem_u32(&aux->fixed_full), n_item & 1, abort_flag, kPolls);
         for (int i = 0; ok && i < g.n_iter; ++i, ++n_stream) {
           const int rs = n_stream % kRing;
           // also when its quarters skip the tile: the wait keeps the issuer from running a whole ring ahead of
           // the other one, whose arrival on empty[rs] must fall into the same phase as this one's
-          ok = mbar_wait(smem_u32(&aux->full[rs]), (n_stream / kRing) & 1, abort_flag);
+          ok = mbar_wait(smem_u32(&aux->full[rs]), (n_stream / kRing) & 1, abort_flag, kPolls);
           if (!ok) break;
 #pragma unroll
           for (int u = 0; u < kQPerIssuer; ++u) {
@@ -290,7 +294,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const int qd = kQPerIssuer * iw + u;
             if (!g.active(qd, i)) continue;
             const int c = cnt[u]++;                 // the quarter's accumulator is reused every time: phase c & 1
-            ok = mbar_wait(smem_u32(&aux->acc_empty[qd]), (c & 1) ^ 1, abort_flag);
+            ok = mbar_wait(smem_u32(&aux->acc_empty[qd]), (c & 1) ^ 1, abort_flag, kPolls);
             if (!ok) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + qd * kTile;
@@ -313,7 +317,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (*abort_flag) {
         // wait (bounded) until every MMA already issued has retired before TMEM and shared memory go away
         umma_commit(smem_u32(&aux->drain[iw]));
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(smem_u32(&aux->drain[iw]), 0); ++i) {}
+        for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(smem_u32(&aux->drain[iw]), 0); ++i) {}
       }
     }
   } else {
@@ -333,7 +337,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     auto epi_sync = [&]() {
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&aux->epi_bar));
-      ok = mbar_wait(smem_u32(&aux->epi_bar), n_esync & 1, abort_flag) && ok;
+      ok = mbar_wait(smem_u32(&aux->epi_bar), n_esync & 1, abort_flag, kPolls) && ok;
       ++n_esync;
     };
     auto release = [&]() {                         // accumulator drained: hand it back to its issuer
@@ -344,7 +348,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
     while (true) {
       const int slot = n_item & 1;
-      ok = mbar_wait(smem_u32(&aux->item_full[slot]), (n_item >> 1) & 1, abort_flag) && ok;
+      ok = mbar_wait(smem_u32(&aux->item_full[slot]), (n_item >> 1) & 1, abort_flag, kPolls) && ok;
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       int it[5];
@@ -384,7 +388,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (!g.active(gi, i)) continue;
             const int c = cnt++;
             const float* lse_buf = aux->lse_chunk[k & 1] + (i & (kLseChunk - 1)) * kTile;
-            ok = mbar_wait(acc_full, c & 1, abort_flag) && ok;
+            ok = mbar_wait(acc_full, c & 1, abort_flag, kPolls) && ok;
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -408,7 +412,7 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         for (int i = 0; i < g.n_iter && ok; ++i) {
           if (!g.active(gi, i)) continue;
           const int c = cnt++;
-          ok = mbar_wait(acc_full, c & 1, abort_flag) && ok;
+          ok = mbar_wait(acc_full, c & 1, abort_flag, kPolls) && ok;
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -462,9 +466,9 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   if (tid == 0 && !dead && *abort_flag) report(a.status, KVCRUSH_DEV_TIMEOUT, kColsum ? KID_SCORE_COLSUM : KID_SCORE_LSE, blockIdx.x, 0);
 }
 
-template <int D, bool kColsum>
-int launch_persist(const CUtensorMap& mq, const CUtensorMap& mk, const PersistArgs& a, int n_sms, cudaStream_t stream) {
-  auto kern = score_persist_kernel<D, kColsum>;
+template <int D, bool kColsum, uint32_t kPolls>
+int launch_persist_polls(const CUtensorMap& mq, const CUtensorMap& mk, const PersistArgs& a, int n_sms, cudaStream_t stream) {
+  auto kern = score_persist_kernel<D, kColsum, kPolls>;
   constexpr int smem = PSmem<D>::kTotal;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return KVCRUSH_ERR_CUDA;
   const int blocks = a.total_items < n_sms ? a.total_items : n_sms;
@@ -472,35 +476,48 @@ int launch_persist(const CUtensorMap& mq, const CUtensorMap& mk, const PersistAr
   return check_launch();
 }
 
+template <int D, bool kColsum>
+int launch_persist(const CUtensorMap& mq, const CUtensorMap& mk, const PersistArgs& a, bool short_waits, int n_sms,
+                   cudaStream_t stream) {
+  return short_waits ? launch_persist_polls<D, kColsum, kShortWaitPolls>(mq, mk, a, n_sms, stream)
+                     : launch_persist_polls<D, kColsum, kWaitPolls>(mq, mk, a, n_sms, stream);
+}
+
 }  // namespace
 
 size_t score_tensor_counter_bytes() { return 256; }
 
-bool score_tensor_supported(const Shape& s, const TensorView& Q, const TensorView& K) {
-  if (Q.dtype != K.dtype || (Q.dtype != KVCRUSH_BF16 && Q.dtype != KVCRUSH_FP16)) return false;
-  if (s.D < 8 || s.D > 128 || s.D % 8 != 0) return false;      // other widths ride in the 64- or 128-wide kernel
-  if (s.T < 1) return false;
-  return encode_fn() != nullptr;
+int score_tensor_plan(const Shape& s, const TensorView& Q, const TensorView& K, ScoreTensorMaps* maps) {
+  static_assert(sizeof(CUtensorMap) == sizeof(maps->q) && alignof(CUtensorMap) <= 64, "tensor map storage");
+  if (Q.dtype != K.dtype || (Q.dtype != KVCRUSH_BF16 && Q.dtype != KVCRUSH_FP16)) return TENSOR_PLAN_NO;
+  if (s.D < 8 || s.D > 128 || s.D % 8 != 0) return TENSOR_PLAN_NO;      // other widths ride in the 64- or 128-wide kernel
+  if (s.T < 1) return TENSOR_PLAN_NO;
+  if (encode_fn() == nullptr) return TENSOR_PLAN_NO_ENCODER;
+  if (!make_map(reinterpret_cast<CUtensorMap*>(maps->q), Q, s.D, s.T, s.Hq, s.n_layers) ||
+      !make_map(reinterpret_cast<CUtensorMap*>(maps->k), K, s.D, s.T, s.Hkv, s.n_layers))
+    return TENSOR_PLAN_NO;                                               // strides or extents the TMA unit cannot take
+  return TENSOR_PLAN_OK;
 }
 
 
-int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView& Q, const TensorView& K,
-                                   float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws,
-                                   int* counters, float* scores, float* lse_out, int normalize, int32_t* status,
-                                   cudaStream_t stream) {
+int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView& Q, const ScoreTensorMaps& maps,
+                        float scale_log2, const float* lse_in, float lse_in_mul, float* lse2_ws,
+                        int* counters, float* scores, float* lse_out, int normalize, int32_t* status,
+                        const ScoreDiag& diag, cudaStream_t stream) {
   static_assert(sizeof(PAux) <= 26624, "aux block too large");
   if (!(scale_log2 > 0.f)) return KVCRUSH_ERR_UNSUPPORTED;
-  CUtensorMap mq, mk;
-  if (!make_map(&mq, Q, s.D, s.T, s.Hq, s.n_layers) || !make_map(&mk, K, s.D, s.T, s.Hkv, s.n_layers))
-    return KVCRUSH_ERR_CUDA;
+  const CUtensorMap& mq = *reinterpret_cast<const CUtensorMap*>(maps.q);
+  const CUtensorMap& mk = *reinterpret_cast<const CUtensorMap*>(maps.k);
   int dev = 0, n_sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sms < 1)
     return KVCRUSH_ERR_CUDA;
   PersistArgs a{};
   a.s = s; a.scale_log2 = scale_log2; a.normalize = normalize; a.bf16 = Q.dtype == KVCRUSH_BF16; a.status = status; a.scores = scores;
+  const bool sw = diag.short_waits != 0;
+  a.withhold_first_item = diag.withhold_first_item;
   a.max_blocks = (s.max_seqlen + kBlockRows - 1) / kBlockRows;
-  // work items per (layer, head): every 256-row block for the column sweep; for the row sweep only the
+  // work items per (layer, head): every 512-row block for the column sweep; for the row sweep only the
   // blocks that hold voting queries
   long long items_col = 0, items_row = 0;
   for (int i = 0; i < s.n_seqs; ++i) {
@@ -517,7 +534,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
   if (!lse_in) {
     a.lse2_out = lse2_ws; a.lse_nat_out = lse_out; a.counter = counters;
     a.n_items = (int)items_row; a.total_items = (int)(items_row * s.n_layers * s.Hq);
-    rc = s.D > 64 ? launch_persist<128, false>(mq, mk, a, n_sms, stream) : launch_persist<64, false>(mq, mk, a, n_sms, stream);
+    rc = s.D > 64 ? launch_persist<128, false>(mq, mk, a, sw, n_sms, stream) : launch_persist<64, false>(mq, mk, a, sw, n_sms, stream);
     if (rc != KVCRUSH_OK) return rc;
     a.lse = lse2_ws; a.lse_mul = 1.f;
   } else {
@@ -525,7 +542,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
   }
   a.counter = counters + 1;
   a.n_items = (int)items_col; a.total_items = (int)(items_col * s.n_layers * s.Hq);
-  return s.D > 64 ? launch_persist<128, true>(mq, mk, a, n_sms, stream) : launch_persist<64, true>(mq, mk, a, n_sms, stream);
+  return s.D > 64 ? launch_persist<128, true>(mq, mk, a, sw, n_sms, stream) : launch_persist<64, true>(mq, mk, a, sw, n_sms, stream);
 }
 
 }  // namespace kvc

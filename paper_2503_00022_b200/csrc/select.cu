@@ -4,6 +4,8 @@
 //                          float64, heads added in ascending order inside each KV group and the
 //                          group sums added in ascending order; stored as an order-preserving
 //                          64-bit key.  One thread per (layer, token), coalesced per-head rows.
+//                          Skipped when the caller hands over I(t) (the signature stage can write it
+//                          from the loads it does anyway).
 //   select_segment_kernel  one CTA per segment:
 //                            1. exact radix select of the B_imp-th largest key, ties admitted in
 //                               ascending token order                         -> important set
@@ -26,6 +28,14 @@ using sel::kWarps;
 using sel::kFull;
 using sel::head_mask;
 constexpr int kMaxBins = 129;              // Hamming distances 0..128
+
+// Order-preserving 64-bit key of a float64 importance; tokens kept by decree (the first keep_initial and the last
+// keep_recent of a sequence of L tokens) rank as +infinity.
+__device__ __forceinline__ unsigned long long importance_key(double v, int t, int L, int keep_initial, int keep_recent) {
+  if (t < keep_initial || t >= L - keep_recent) v = __longlong_as_double(0x7FF0000000000000LL);
+  const unsigned long long b = (unsigned long long)__double_as_longlong(v);
+  return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+}
 
 __global__ void __launch_bounds__(256)
 importance_kernel(Shape s, const float* __restrict__ scores, int keep_initial, int keep_recent,
@@ -51,17 +61,32 @@ importance_kernel(Shape s, const float* __restrict__ scores, int keep_initial, i
     }
   }
   total = __dadd_rn(total, 0.0);           // -0.0 -> +0.0
+  int t = 0, L = 0x7FFFFFFF;
   if (keep_recent > 0 || keep_initial > 0) {   // the first / last tokens of a sequence are important by decree
     const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
-    if (tok >= __ldg(s.cu_seqlens + seq + 1) - keep_recent || tok < __ldg(s.cu_seqlens + seq) + keep_initial)
-      total = __longlong_as_double(0x7FF0000000000000LL);
+    t = tok - __ldg(s.cu_seqlens + seq);
+    L = __ldg(s.cu_seqlens + seq + 1) - __ldg(s.cu_seqlens + seq);
   }
-  const unsigned long long b = (unsigned long long)__double_as_longlong(total);
-  keys[gid] = (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+  keys[gid] = importance_key(total, t, L, keep_initial, keep_recent);
+}
+
+// Keys from an importance array the caller supplies (segments too long for the shared-memory copy, where the
+// conversion happens otherwise).
+__global__ void __launch_bounds__(256)
+importance_keys_kernel(Shape s, const double* __restrict__ imp, int keep_initial, int keep_recent,
+                       unsigned long long* __restrict__ keys) {
+  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= (long long)s.n_layers * s.T) return;
+  const int tok = (int)(gid % s.T);
+  const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
+  const int t0 = __ldg(s.cu_seqlens + seq);
+  keys[gid] = importance_key(imp[gid], tok - t0, __ldg(s.cu_seqlens + seq + 1) - t0, keep_initial, keep_recent);
 }
 
 struct SelectArgs {
-  const unsigned long long* keys;     // [n_layers][T]
+  const unsigned long long* keys;     // [n_layers][T] importance keys; or, when NULL,
+  const double* imp;                  // [n_layers][T] importance values, turned into keys while they are staged
+  int keep_initial, keep_recent;      // tokens important by decree (applied with imp; keys have them built in)
   const uint32_t* sigs;               // [n_layers][T][W]
   const int32_t* budget_imp;
   const int32_t* budget_rep;
@@ -71,6 +96,7 @@ struct SelectArgs {
   const int32_t* cu_kept;
   int32_t* idx;
   uint8_t* kind;
+  int32_t* n_kept;                    // optional [n_layers][n_seqs]: tokens kept per segment
   int32_t* sorted;                    // [n_layers][T] scratch: grouped tokens in (d, t) order
   int mask_words;                     // words of one membership mask in shared memory
   int stage_words;                    // max_seqlen rounded up to a multiple of 4 (one staged int32 per token)
@@ -101,6 +127,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
   int32_t* out_idx = a.idx + __ldg(a.cu_kept + seg);
   uint8_t* out_kind = a.kind ? a.kind + __ldg(a.cu_kept + seg) : nullptr;
 
+  if (a.n_kept && tid == 0) a.n_kept[seg] = (int)min((long long)b_imp + b_rep, (long long)L);
   if ((long long)b_imp + b_rep >= L) {             // budget covers the sequence: keep everything
     for (int i = tid; i < L; i += kThreads) {
       out_idx[i] = i;
@@ -112,7 +139,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
   // The segment's arrays are read many times with dependent addresses (8 radix sweeps, two counting-sort
   // sweeps, one gather per bucket), so whatever fits is first copied into shared memory; the rest is read
   // through L2.  The pointers below are generic and point to either place.
-  const unsigned long long* keys = a.keys + (size_t)layer * s.T + t0;
+  const unsigned long long* keys = a.keys ? a.keys + (size_t)layer * s.T + t0 : nullptr;
   const uint32_t* sig = a.sigs + ((size_t)layer * s.T + t0) * W;
   int32_t* sorted = a.sorted + (size_t)layer * s.T + t0;
   {
@@ -125,7 +152,12 @@ select_segment_kernel(Shape s, SelectArgs a) {
     }
     if (a.stage_keys) {
       unsigned long long* ks = reinterpret_cast<unsigned long long*>(arena);
-      for (int i = tid; i < L; i += kThreads) ks[i] = keys[i];
+      if (a.keys) {
+        for (int i = tid; i < L; i += kThreads) ks[i] = keys[i];
+      } else {
+        const double* imp = a.imp + (size_t)layer * s.T + t0;
+        for (int i = tid; i < L; i += kThreads) ks[i] = importance_key(imp[i], i, L, a.keep_initial, a.keep_recent);
+      }
       keys = ks;
     }
   }
@@ -319,28 +351,44 @@ size_t select_workspace_bytes(const Shape& s) {
   return ((n * 8 + 255) / 256) * 256 + ((n * 4 + 255) / 256) * 256;
 }
 
-int launch_select(const Shape& s, const float* scores, const uint32_t* sigs, const int32_t* budget_imp,
+int launch_select(const Shape& s, const float* scores, const double* importance, const uint32_t* sigs,
+                  const int32_t* budget_imp,
                   const int32_t* budget_rep, int anchor_mode, const uint32_t* anchor_bits, int anchor_per_segment,
-                  int keep_initial, int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind, void* ws,
-                  cudaStream_t stream) {
-  if (s.T == 0) return KVCRUSH_OK;
+                  int keep_initial, int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind,
+                  int32_t* n_kept, void* ws, cudaStream_t stream) {
+  if (s.T == 0) {                                   // nothing but empty sequences: every segment keeps nothing
+    if (n_kept && cudaMemsetAsync(n_kept, 0, (size_t)s.n_layers * s.n_seqs * sizeof(int32_t), stream) != cudaSuccess)
+      return KVCRUSH_ERR_CUDA;
+    return KVCRUSH_OK;
+  }
   const size_t n = (size_t)s.n_layers * s.T;
   unsigned long long* keys = static_cast<unsigned long long*>(ws);
   int32_t* sorted = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(ws) + ((n * 8 + 255) / 256) * 256);
-  if (launch_importance(s, scores, keep_initial, keep_recent, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
 
   SelectArgs a{};
-  a.keys = keys; a.sigs = sigs; a.budget_imp = budget_imp; a.budget_rep = budget_rep;
+  a.sigs = sigs; a.budget_imp = budget_imp; a.budget_rep = budget_rep;
   a.anchor_mode = anchor_mode; a.anchor_bits = anchor_bits; a.anchor_per_segment = anchor_per_segment;
-  a.cu_kept = cu_kept; a.idx = idx; a.kind = kind; a.sorted = sorted;
+  a.cu_kept = cu_kept; a.idx = idx; a.kind = kind; a.n_kept = n_kept; a.sorted = sorted;
   a.mask_words = ((s.max_seqlen + 31) / 32 + 3) & ~3;
   a.stage_words = (s.max_seqlen + 3) & ~3;
   size_t dyn = (size_t)a.mask_words * 2 * sizeof(uint32_t);
-  const size_t budget = 196 * 1024;     // dynamic shared memory this kernel may take (static part: ~19 KB)
+  const size_t budget = 196 * 1024;     // dynamic shared memory this kernel may take (static part: ~27 KB)
   const size_t per_tok = (size_t)a.stage_words * sizeof(uint32_t);
   if (dyn + per_tok <= budget) { a.stage_sorted = 1; dyn += per_tok; }
   if (dyn + per_tok * s.W <= budget) { a.stage_sig = 1; dyn += per_tok * s.W; }
   if (dyn + 2 * per_tok <= budget) { a.stage_keys = 1; dyn += 2 * per_tok; }
+  // importance keys: computed here from the scores, or taken from the caller's I(t) - converted while the segment
+  // kernel stages them, or by a small kernel when the segments are too long to be staged
+  if (!importance) {
+    if (launch_importance(s, scores, keep_initial, keep_recent, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+    a.keys = keys;
+  } else if (a.stage_keys) {
+    a.imp = importance; a.keep_initial = keep_initial; a.keep_recent = keep_recent;
+  } else {
+    importance_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, importance, keep_initial, keep_recent, keys);
+    if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+    a.keys = keys;
+  }
   if (dyn > 16 * 1024) {     // static + dynamic shared memory above the 48 KB default needs the opt-in
     cudaError_t e = cudaSuccess;
     switch (s.W) {

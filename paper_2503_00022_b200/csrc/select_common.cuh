@@ -1,5 +1,6 @@
-// Block-wide building blocks shared by the token-level and the page-level selection kernels:
-// exact top-k marking of 64-bit keys and emission of the kept set from two membership masks.
+// Block-wide building blocks shared by the signature, the token-level and the page-level selection kernels:
+// the search for the k-th largest key by radix histograms, exact top-k marking of 64-bit keys and emission of
+// the kept set from two membership masks.
 #pragma once
 
 #include "common.cuh"
@@ -10,11 +11,17 @@ namespace sel {
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kDigitBits = 11;                 // radix digit of the 64-bit selection
+constexpr int kBins = 1 << kDigitBits;
+constexpr int kSmallList = 32;                 // candidates one warp ranks directly
 
 struct Scratch {
-  uint32_t hist[256];
-  unsigned long long sel_prefix;
-  uint32_t sel_k;
+  uint32_t hist[kBins];
+  unsigned long long red[2][kWarps];           // per-warp minimum / maximum
+  unsigned long long small[kSmallList];
+  unsigned long long sel_x;                    // result of a search step
+  uint32_t sel[3];                             // digit, remaining rank, live keys
+  uint32_t small_n;
   int warp_tot[kWarps];
 };
 
@@ -31,71 +38,139 @@ __device__ __forceinline__ void warp_range(int n, int warp, int& r_lo, int& r_hi
   r_hi = min(n, r_lo + per_warp);
 }
 
+// The digit that holds the k_rem-th largest key, from a complete histogram of one digit position (bins in
+// ascending digit order, counted from the top): out[0] = digit, out[1] = rank left inside that digit's bin,
+// out[2] = keys in the bin.  Called by all kT threads of the block; k_rem is at most the histogram's total.
+// The histogram must be complete (a barrier lies between its last update and this call); the result is
+// visible to every thread on return.
+template <int kT>
+__device__ __forceinline__ void find_digit_desc(const uint32_t* hist, int n_bins, uint32_t k_rem, int* warp_tot,
+                                                uint32_t* out) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per = n_bins >= kT ? n_bins / kT : 1;           // bins per thread, walked from the top digit down
+  const int n_act = n_bins / per;
+  uint32_t local = 0;
+  if (tid < n_act)
+    for (int j = 0; j < per; ++j) local += hist[n_bins - 1 - (tid * per + j)];
+  uint32_t incl = local;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t v = __shfl_up_sync(kFull, incl, d);
+    if (lane >= d) incl += v;
+  }
+  if (lane == 31) warp_tot[warp] = (int)incl;
+  __syncthreads();
+  uint32_t excl = incl - local;
+  for (int w = 0; w < warp; ++w) excl += (uint32_t)warp_tot[w];
+  if (tid < n_act && excl < k_rem && k_rem <= excl + local) {
+    uint32_t acc = excl;
+    for (int j = 0; j < per; ++j) {
+      const int bin = n_bins - 1 - (tid * per + j);
+      const uint32_t c = hist[bin];
+      if (k_rem <= acc + c) {
+        out[0] = (uint32_t)bin; out[1] = k_rem - acc; out[2] = c;
+        break;
+      }
+      acc += c;
+    }
+  }
+  __syncthreads();
+}
+
+// One warp ranks at most 32 candidates held one per lane (lanes >= n hold nothing): returns in every lane the
+// k_rem-th largest value and sets k_out to the rank left among the candidates equal to it.
+__device__ __forceinline__ unsigned long long warp_rank_select(unsigned long long v, int n, uint32_t k_rem, int lane,
+                                                               uint32_t& k_out) {
+  uint32_t gt = 0, ge = 0;
+  for (int j = 0; j < n; ++j) {
+    const unsigned long long o = __shfl_sync(kFull, v, j);
+    gt += o > v;
+    ge += o >= v;
+  }
+  const bool hit = lane < n && gt < k_rem && k_rem <= ge;
+  const unsigned who = __ballot_sync(kFull, hit);
+  const int src = __ffs(who) - 1;                     // equal candidates all qualify: any of them
+  k_out = k_rem - __shfl_sync(kFull, gt, src);
+  return __shfl_sync(kFull, v, src);
+}
+
 // Sets bit i of imp_mask for the k items with the largest keys[0..n); equal keys are admitted in ascending
-// index order.  Exact MSB-first radix select (8 digits of 8 bits), then one ordered pass.  Called by all
-// threads of the block; imp_mask must be zero on entry; 0 < k < n.
+// index order.  Exact: the k-th largest key is found by radix histograms over (key - smallest key), starting at
+// the top bit in which the keys of this segment differ at all - the digits are then spread over the bins whatever
+// the keys' common magnitude -, and as soon as at most 32 candidates are left one warp ranks them directly; then
+// one ordered pass marks the members.  Called by all threads of the block; imp_mask must be zero on entry;
+// 0 < k < n.
 __device__ __forceinline__ void mark_top_keys(const unsigned long long* keys, int n, int k, uint32_t* imp_mask,
                                               Scratch& sc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned lt_mask = (1u << lane) - 1u;
   int r_lo, r_hi;
   warp_range(n, warp, r_lo, r_hi);
-  unsigned long long prefix = 0;
-  uint32_t k_rem = k;
-  for (int shift = 56; shift >= 0; shift -= 8) {
-    for (int i = tid; i < 256; i += kThreads) sc.hist[i] = 0;
-    __syncthreads();
-    const unsigned long long hi_mask = shift == 56 ? 0ull : (~0ull << (shift + 8));
-    for (int base = 0; base < n; base += kThreads) {
-      const int i = base + tid;
-      const bool in = i < n;
-      const unsigned long long key = in ? keys[i] : 0ull;
-      const bool live = in && ((key & hi_mask) == prefix);
-      const uint32_t digit = (uint32_t)(key >> shift) & 0xFFu;
-      // high digits (sign, exponent) are the same for almost every key: one add per warp then;
-      // low digits are spread over the 256 bins, where plain shared-memory atomics do not collide much
-      const unsigned voters = __ballot_sync(kFull, live);
-      if (voters) {
-        const uint32_t d0 = __shfl_sync(kFull, digit, __ffs(voters) - 1);
-        if (__all_sync(kFull, !live || digit == d0)) {
-          if (lane == 0) atomicAdd(&sc.hist[d0], __popc(voters));
-        } else if (live) {
-          atomicAdd(&sc.hist[digit], 1u);
-        }
-      }
-    }
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t local = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) local += sc.hist[255 - 8 * lane - j];
-      uint32_t incl = local;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(kFull, incl, d);
-        if (lane >= d) incl += v;
-      }
-      const uint32_t excl = incl - local;
-      if (excl < k_rem && k_rem <= incl) {
-        uint32_t acc = excl;
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t c = sc.hist[255 - 8 * lane - j];
-          if (k_rem <= acc + c) {
-            sc.sel_prefix = prefix | ((unsigned long long)(255 - 8 * lane - j) << shift);
-            sc.sel_k = k_rem - acc;
-            break;
-          }
-          acc += c;
-        }
-      }
-    }
-    __syncthreads();
-    prefix = sc.sel_prefix;
-    k_rem = sc.sel_k;
-    __syncthreads();
+
+  // smallest and largest key
+  unsigned long long lo = ~0ull, hi = 0ull;
+  for (int i = tid; i < n; i += kThreads) {
+    const unsigned long long key = keys[i];
+    lo = key < lo ? key : lo;
+    hi = key > hi ? key : hi;
   }
-  // prefix = the k-th largest key; k_rem = how many keys equal to it are admitted
-  const unsigned long long kth = prefix;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    const unsigned long long a = __shfl_xor_sync(kFull, lo, d), b = __shfl_xor_sync(kFull, hi, d);
+    lo = a < lo ? a : lo;
+    hi = b > hi ? b : hi;
+  }
+  if (lane == 0) { sc.red[0][warp] = lo; sc.red[1][warp] = hi; }
+  __syncthreads();
+  lo = sc.red[0][lane];
+  hi = sc.red[1][lane];
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    const unsigned long long a = __shfl_xor_sync(kFull, lo, d), b = __shfl_xor_sync(kFull, hi, d);
+    lo = a < lo ? a : lo;
+    hi = b > hi ? b : hi;
+  }
+  const unsigned long long base = lo, range = hi - lo;
+
+  // x = key - base has `rem` significant bits; `top` is the value of the bits of x above them chosen so far
+  int rem = range ? 64 - __clzll((long long)range) : 0;
+  unsigned long long top = 0;
+  uint32_t k_rem = (uint32_t)k;
+  while (rem > 0) {
+    const int w = rem < kDigitBits ? rem : kDigitBits, shift = rem - w, n_bins = 1 << w;
+    for (int i = tid; i < n_bins; i += kThreads) sc.hist[i] = 0;
+    if (tid == 0) sc.small_n = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += kThreads) {
+      const unsigned long long x = keys[i] - base;
+      if (((x >> 1) >> (rem - 1)) == top) atomicAdd(&sc.hist[(uint32_t)(x >> shift) & (uint32_t)(n_bins - 1)], 1u);
+    }
+    __syncthreads();
+    find_digit_desc<kThreads>(sc.hist, n_bins, k_rem, sc.warp_tot, sc.sel);
+    top = (top << w) | sc.sel[0];
+    k_rem = sc.sel[1];
+    const uint32_t live = sc.sel[2];
+    rem = shift;
+    if (rem > 0 && live <= (uint32_t)kSmallList) {     // few candidates: one warp ranks their remaining bits
+      for (int i = tid; i < n; i += kThreads) {
+        const unsigned long long x = keys[i] - base;
+        if (((x >> 1) >> (rem - 1)) == top) sc.small[atomicAdd(&sc.small_n, 1u)] = x;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        uint32_t k_out;
+        const unsigned long long v = warp_rank_select(lane < (int)live ? sc.small[lane] : 0ull, (int)live, k_rem, lane, k_out);
+        if (lane == 0) { sc.sel_x = v; sc.sel[1] = k_out; }
+      }
+      __syncthreads();
+      top = sc.sel_x;
+      k_rem = sc.sel[1];
+      rem = 0;
+    }
+    __syncthreads();                                   // sc.sel and sc.hist are rewritten by the next step
+  }
+  // kth = the k-th largest key; k_rem = how many keys equal to it are admitted
+  const unsigned long long kth = base + top;
   int n_eq = 0;
   for (int i = r_lo + lane; i < r_hi; i += 32) n_eq += (keys[i] == kth);
 #pragma unroll
@@ -104,14 +179,14 @@ __device__ __forceinline__ void mark_top_keys(const unsigned long long* keys, in
   __syncthreads();
   int eq_before = 0;
   for (int w = 0; w < warp; ++w) eq_before += sc.warp_tot[w];
-  for (int base = r_lo; base < r_hi; base += 32) {
-    const int i = base + lane;
+  for (int base_i = r_lo; base_i < r_hi; base_i += 32) {
+    const int i = base_i + lane;
     const unsigned long long key = i < r_hi ? keys[i] : 0ull;
     const bool eq = i < r_hi && key == kth;
     const unsigned eq_b = __ballot_sync(kFull, eq);
     const bool imp = i < r_hi && (key > kth || (eq && (uint32_t)(eq_before + __popc(eq_b & lt_mask)) < k_rem));
     const unsigned imp_b = __ballot_sync(kFull, imp);
-    if (lane == 0) imp_mask[base >> 5] = imp_b;
+    if (lane == 0) imp_mask[base_i >> 5] = imp_b;
     eq_before += __popc(eq_b);
   }
   __syncthreads();

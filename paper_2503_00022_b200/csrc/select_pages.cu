@@ -25,7 +25,8 @@ using sel::kFull;
 using sel::head_mask;
 
 struct PageArgs {
-  const unsigned long long* tok_keys;  // [n_layers][T] order-preserving keys of I(t)
+  const unsigned long long* tok_keys;  // [n_layers][T] order-preserving keys of I(t); or, when NULL,
+  const double* tok_imp;               // [n_layers][T] I(t) itself, handed over by the caller
   const uint32_t* sigs;                // [n_layers][T][W]
   const int32_t* budget_imp;
   const int32_t* budget_rep;
@@ -35,6 +36,7 @@ struct PageArgs {
   const int32_t* cu_kept;
   int32_t* page_idx;
   uint8_t* kind;
+  int32_t* n_kept;                     // optional [n_layers][n_seqs]: pages kept per segment
   int P;                               // tokens per page
   int PW;                              // words per page vector = P * W
   int np_cap;                          // capacity of the per-page arrays (pages, multiple of 32)
@@ -77,6 +79,7 @@ select_pages_kernel(Shape s, PageArgs a) {
   int32_t* out_idx = a.page_idx + __ldg(a.cu_kept + seg);
   uint8_t* out_kind = a.kind ? a.kind + __ldg(a.cu_kept + seg) : nullptr;
 
+  if (a.n_kept && tid == 0) a.n_kept[seg] = (int)min((long long)b_imp + b_rep, (long long)n_pages);
   if ((long long)b_imp + b_rep >= n_pages) {       // budget covers the sequence: keep every page
     for (int i = tid; i < n_pages; i += kThreads) {
       out_idx[i] = i;
@@ -85,7 +88,8 @@ select_pages_kernel(Shape s, PageArgs a) {
     return;
   }
 
-  const unsigned long long* tkeys = a.tok_keys + (size_t)layer * s.T + t0;
+  const unsigned long long* tkeys = a.tok_keys ? a.tok_keys + (size_t)layer * s.T + t0 : nullptr;
+  const double* timp = a.tok_imp ? a.tok_imp + (size_t)layer * s.T + t0 : nullptr;
   const uint32_t* sig = a.sigs + ((size_t)layer * s.T + t0) * W;
   const int n_words = (n_pages + 31) >> 5;
 
@@ -94,12 +98,13 @@ select_pages_kernel(Shape s, PageArgs a) {
     const int first = p * P, n_tok = min(P, L - first);
     double acc = 0.0;
     for (int i0 = 0; i0 < n_tok; i0 += 8) {        // the adds are sequential by definition, the loads are not
-      unsigned long long kk[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) kk[j] = i0 + j < n_tok ? tkeys[first + i0 + j] : 0ull;
+      double vv[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        if (i0 + j < n_tok) acc = __dadd_rn(acc, key_to_double(kk[j]));
+        vv[j] = i0 + j >= n_tok ? 0.0 : timp ? timp[first + i0 + j] : key_to_double(tkeys[first + i0 + j]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (i0 + j < n_tok) acc = __dadd_rn(acc, vv[j]);
     }
     if (p < a.keep_initial || p >= n_pages - a.keep_recent) acc = __longlong_as_double(0x7FF0000000000000LL);
     pkeys[p] = double_to_key(acc);
@@ -235,18 +240,24 @@ select_pages_kernel(Shape s, PageArgs a) {
 
 }  // namespace
 
-int launch_select_pages(const Shape& s, const float* scores, const uint32_t* sigs, int page_size,
+int launch_select_pages(const Shape& s, const float* scores, const double* importance, const uint32_t* sigs,
+                        int page_size,
                         const int32_t* budget_imp, const int32_t* budget_rep, int anchor_mode,
                         const uint32_t* anchor_bits, int anchor_per_segment, int keep_initial, int keep_recent,
-                        const int32_t* cu_kept, int32_t* page_idx, uint8_t* kind, void* ws, cudaStream_t stream) {
-  if (s.T == 0) return KVCRUSH_OK;
+                        const int32_t* cu_kept, int32_t* page_idx, uint8_t* kind, int32_t* n_kept, void* ws,
+                        cudaStream_t stream) {
+  if (s.T == 0) {                                   // nothing but empty sequences: every segment keeps nothing
+    if (n_kept && cudaMemsetAsync(n_kept, 0, (size_t)s.n_layers * s.n_seqs * sizeof(int32_t), stream) != cudaSuccess)
+      return KVCRUSH_ERR_CUDA;
+    return KVCRUSH_OK;
+  }
   unsigned long long* keys = static_cast<unsigned long long*>(ws);
-  if (launch_importance(s, scores, 0, 0, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+  if (!importance && launch_importance(s, scores, 0, 0, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
 
   PageArgs a{};
-  a.tok_keys = keys; a.sigs = sigs; a.budget_imp = budget_imp; a.budget_rep = budget_rep;
+  a.tok_keys = importance ? nullptr : keys; a.tok_imp = importance; a.sigs = sigs; a.budget_imp = budget_imp; a.budget_rep = budget_rep;
   a.anchor_mode = anchor_mode; a.anchor_bits = anchor_bits; a.anchor_per_segment = anchor_per_segment;
-  a.cu_kept = cu_kept; a.page_idx = page_idx; a.kind = kind;
+  a.cu_kept = cu_kept; a.page_idx = page_idx; a.kind = kind; a.n_kept = n_kept;
   a.P = page_size; a.PW = page_size * s.W;
   a.keep_initial = keep_initial; a.keep_recent = keep_recent;
   const int max_pages = (s.max_seqlen + page_size - 1) / page_size;
@@ -255,7 +266,7 @@ int launch_select_pages(const Shape& s, const float* scores, const uint32_t* sig
   while (a.sort_cap < a.np_cap) a.sort_cap <<= 1;
   const size_t fixed = (size_t)a.np_cap * 8 + (size_t)a.sort_cap * 4 + (size_t)a.np_cap / 32 * 8 + (size_t)a.PW * 4;
   const size_t per_worker = (size_t)a.PW * 32 * sizeof(unsigned short);
-  const size_t budget = 220 * 1024;       // dynamic shared memory this kernel may take (static part: ~1.2 KB)
+  const size_t budget = 212 * 1024;       // dynamic shared memory this kernel may take (static part: ~10 KB)
   a.n_workers = (int)((budget - fixed) / per_worker);
   if (a.n_workers > sel::kWarps) a.n_workers = sel::kWarps;
   if (a.n_workers < 2) return KVCRUSH_ERR_UNSUPPORTED;

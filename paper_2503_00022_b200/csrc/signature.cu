@@ -1,18 +1,26 @@
 // Stage 2: per-head thresholds and packed binary signatures (Algorithm 1 and Sec. 3.1 of the paper).
 //
-//   theta_select_kernel   theta = keep-th largest score of one (layer, sequence, head): an exact
-//                         MSB-first radix select over order-preserving 32-bit keys (4 sweeps of 8
-//                         bits, shared-memory histograms with a one-add-per-warp path for uniform digits).
-//   binarise_pack_kernel  one thread per (layer, token): compares the token's score of every head
-//                         with that head's threshold and packs the bits.  Lanes are consecutive
-//                         tokens, so every per-head load is a coalesced 128-byte row.
-#include "common.cuh"
+//   theta_select_kernel       theta = keep-th largest score of one (layer, sequence, head) row of up to 32768
+//                             tokens: the row is read once into registers as order-preserving 32-bit keys, and
+//                             the k-th largest is found by 12-bit radix histograms over (key - smallest key),
+//                             starting at the top bit in which the row's keys differ at all; one warp ranks the
+//                             last few candidates directly.  Usually one histogram pass.
+//   theta_stream_kernel       the same result for longer rows: MSB-first radix select (4 sweeps of 8 bits) that
+//                             re-reads the row from memory (or from a shared-memory copy) in every sweep.
+//   signature_pack_kernel     one thread per (layer, token): loads the token's score of every head (32 loads in
+//                             flight), compares with that head's threshold and packs the bits; from the same
+//                             loads it can add up the token's importance I(t) in float64, in the fixed order
+//                             stage 3 defines, which saves stage 3 its own pass over the scores.
+//                             Lanes are consecutive tokens, so every per-head load is a coalesced 128-byte row.
+#include "select_common.cuh"
 
 namespace kvc {
 
 namespace {
 
 constexpr int kSelectThreads = 512;
+constexpr int kThetaBits = 12;                 // radix digit of theta_select_kernel
+constexpr int kThetaBins = 1 << kThetaBits;
 
 // float -> uint32 such that a < b  <=>  key(a) < key(b) (for non-NaN values)
 __device__ __forceinline__ uint32_t order_key(float x) {
@@ -23,8 +31,92 @@ __device__ __forceinline__ float key_to_float(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
-__global__ void __launch_bounds__(kSelectThreads)
+// kT threads, each holding up to kItems keys of the row: rows of up to kT * kItems tokens.
+template <int kT, int kItems>
+__global__ void __launch_bounds__(kT)
 theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __restrict__ sig_keep,
+                    float* __restrict__ theta) {
+  __shared__ uint32_t hist[kThetaBins];
+  __shared__ uint32_t red[2][32];
+  __shared__ uint32_t small[sel::kSmallList];
+  __shared__ uint32_t small_n, sel_x;
+  __shared__ uint32_t found[3];
+  __shared__ int warp_tot[32];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int h = blockIdx.x % s.Hq;
+  const int seg = blockIdx.x / s.Hq;              // layer * n_seqs + seq
+  const int layer = seg / s.n_seqs, seq = seg - layer * s.n_seqs;
+  const int t0 = __ldg(s.cu_seqlens + seq);
+  const int L = __ldg(s.cu_seqlens + seq + 1) - t0;
+  const int keep = __ldg(sig_keep + seg);
+  float* out = theta + (size_t)seg * s.Hq + h;
+  if (keep <= 0 || keep >= L) {
+    if (tid == 0) *out = keep <= 0 ? __int_as_float(0x7F800000) : __int_as_float(0xFF800000);
+    return;
+  }
+  const float* row = scores + ((size_t)layer * s.Hq + h) * s.T + t0;
+
+  uint32_t key[kItems];
+  uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+#pragma unroll
+  for (int j = 0; j < kItems; ++j) {
+    const int i = j * kT + tid;
+    key[j] = i < L ? order_key(__ldg(row + i)) : 0u;
+  }
+#pragma unroll
+  for (int j = 0; j < kItems; ++j)
+    if (j * kT + tid < L) { lo = min(lo, key[j]); hi = max(hi, key[j]); }
+  lo = __reduce_min_sync(sel::kFull, lo);
+  hi = __reduce_max_sync(sel::kFull, hi);
+  if (lane == 0) { red[0][warp] = lo; red[1][warp] = hi; }
+  __syncthreads();
+  lo = __reduce_min_sync(sel::kFull, lane < kT / 32 ? red[0][lane] : 0xFFFFFFFFu);
+  hi = __reduce_max_sync(sel::kFull, lane < kT / 32 ? red[1][lane] : 0u);
+  const uint32_t base = lo, range = hi - lo;
+
+  // x = key - base has `rem` significant bits; `top` is the value of the bits of x above them chosen so far
+  int rem = range ? 32 - __clz(range) : 0;
+  uint32_t top = 0, k_rem = (uint32_t)keep;
+  while (rem > 0) {
+    const int w = rem < kThetaBits ? rem : kThetaBits, shift = rem - w, n_bins = 1 << w;
+    for (int i = tid; i < n_bins; i += kT) hist[i] = 0;
+    if (tid == 0) small_n = 0;
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) {
+      const uint32_t x = key[j] - base;
+      if (j * kT + tid < L && ((x >> 1) >> (rem - 1)) == top) atomicAdd(&hist[(x >> shift) & (uint32_t)(n_bins - 1)], 1u);
+    }
+    __syncthreads();
+    sel::find_digit_desc<kT>(hist, n_bins, k_rem, warp_tot, found);
+    top = (top << w) | found[0];
+    k_rem = found[1];
+    const uint32_t live = found[2];
+    rem = shift;
+    if (rem > 0 && live <= (uint32_t)sel::kSmallList) {     // few candidates: one warp ranks their remaining bits
+#pragma unroll
+      for (int j = 0; j < kItems; ++j) {
+        const uint32_t x = key[j] - base;
+        if (j * kT + tid < L && ((x >> 1) >> (rem - 1)) == top) small[atomicAdd(&small_n, 1u)] = x;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        uint32_t k_out;
+        const unsigned long long v = sel::warp_rank_select(lane < (int)live ? small[lane] : 0u, (int)live, k_rem, lane, k_out);
+        if (lane == 0) sel_x = (uint32_t)v;
+      }
+      __syncthreads();
+      top = sel_x;
+      rem = 0;
+    }
+    __syncthreads();                                         // hist and found are rewritten by the next step
+  }
+  if (tid == 0) *out = key_to_float(base + top);
+}
+
+__global__ void __launch_bounds__(kSelectThreads)
+theta_stream_kernel(Shape s, const float* __restrict__ scores, const int32_t* __restrict__ sig_keep,
                     float* __restrict__ theta, int stage_row) {
   extern __shared__ uint32_t row_keys[];          // the row's order keys when it fits (stage_row), else unused
   __shared__ uint32_t hist[256];
@@ -111,47 +203,93 @@ theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __
   if (threadIdx.x == 0) *out = key_to_float(prefix);
 }
 
-__global__ void __launch_bounds__(256)
-binarise_pack_kernel(Shape s, const float* __restrict__ scores, const float* __restrict__ theta,
-                     uint32_t* __restrict__ sigs) {
-  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (gid >= (long long)s.n_layers * s.T) return;
-  const int layer = (int)(gid / s.T), tok = (int)(gid - (long long)layer * s.T);
-  const int seq = seq_of_token(s.cu_seqlens, s.n_seqs, tok);
+// kImportance: also write I(t) = sum of the token's per-head scores (float64; heads ascending inside each KV
+// group, then the group sums ascending: sequential IEEE additions, so the value is bit-reproducible).
+// Grid: (token blocks, layers).  The thresholds of the block's sequence sit in shared memory when all its tokens
+// belong to one sequence (always, with one sequence per batch); else every thread reads its own sequence's row.
+template <bool kImportance>
+__global__ void __launch_bounds__(256, 3)
+signature_pack_kernel(Shape s, const float* __restrict__ scores, const float* __restrict__ theta,
+                      uint32_t* __restrict__ sigs, double* __restrict__ importance) {
+  __shared__ float th_sh[128];
+  const int layer = blockIdx.y;
+  const int tok0 = blockIdx.x * 256, tok = tok0 + threadIdx.x;
+  const int seq0 = seq_of_token(s.cu_seqlens, s.n_seqs, tok0);
+  const bool one_seq = min(tok0 + 256, s.T) <= __ldg(s.cu_seqlens + seq0 + 1);
+  if (one_seq) {
+    if (threadIdx.x < s.Hq) th_sh[threadIdx.x] = __ldg(theta + ((size_t)layer * s.n_seqs + seq0) * s.Hq + threadIdx.x);
+    __syncthreads();
+  }
+  if (tok >= s.T) return;
+  const float* th = one_seq ? th_sh
+                            : theta + ((size_t)layer * s.n_seqs + seq_of_token(s.cu_seqlens, s.n_seqs, tok)) * s.Hq;
   const float* sc = scores + (size_t)layer * s.Hq * s.T + tok;
-  const float* th = theta + ((size_t)layer * s.n_seqs + seq) * s.Hq;
   uint32_t* out = sigs + ((size_t)layer * s.T + tok) * s.W;
+  double total = 0.0, group = 0.0;
+  int in_group = 0;
   for (int w = 0; w < s.W; ++w) {
     uint32_t word = 0;
-    const int h_end = min(32, s.Hq - 32 * w);
-    for (int b = 0; b < h_end; ++b) {
-      const int h = 32 * w + b;
-      word |= (uint32_t)(__ldg(sc + (size_t)h * s.T) >= __ldg(th + h)) << b;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {             // 16 loads in flight at a time
+      const int h0 = 32 * w + 16 * half;
+      float v[16];
+#pragma unroll
+      for (int b = 0; b < 16; ++b) v[b] = h0 + b < s.Hq ? __ldg(sc + (size_t)(h0 + b) * s.T) : 0.f;
+#pragma unroll
+      for (int b = 0; b < 16; ++b)
+        if (h0 + b < s.Hq) word |= (uint32_t)(v[b] >= th[h0 + b]) << (16 * half + b);
+      if constexpr (kImportance) {
+#pragma unroll
+        for (int b = 0; b < 16; ++b) {
+          if (h0 + b < s.Hq) {
+            group = __dadd_rn(group, (double)v[b]);
+            if (++in_group == s.G) { total = __dadd_rn(total, group); group = 0.0; in_group = 0; }
+          }
+        }
+      }
     }
     out[w] = word;
   }
+  if constexpr (kImportance) importance[(size_t)layer * s.T + tok] = __dadd_rn(total, 0.0);       // -0.0 -> +0.0
+}
+
+template <int kT, int kItems>
+void launch_theta(const Shape& s, const float* scores, const int32_t* sig_keep, float* theta, unsigned blocks,
+                  cudaStream_t stream) {
+  theta_select_kernel<kT, kItems><<<blocks, kT, 0, stream>>>(s, scores, sig_keep, theta);
 }
 
 }  // namespace
 
 int launch_signature(const Shape& s, const float* scores, const int32_t* sig_keep, const float* theta_in,
-                     uint32_t* sigs, float* theta, cudaStream_t stream) {
+                     uint32_t* sigs, float* theta, double* importance, cudaStream_t stream) {
   if (s.T == 0) return KVCRUSH_OK;
   const float* th = theta_in;
   if (!theta_in) {
     const unsigned blocks = (unsigned)s.n_layers * s.n_seqs * s.Hq;
-    const size_t row_bytes = (size_t)s.max_seqlen * sizeof(uint32_t);
-    const int stage_row = row_bytes <= 96 * 1024;
-    const size_t dyn = stage_row ? row_bytes : 0;
-    if (dyn > 40 * 1024 &&
-        cudaFuncSetAttribute(theta_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
-      return KVCRUSH_ERR_CUDA;
-    theta_select_kernel<<<blocks, kSelectThreads, dyn, stream>>>(s, scores, sig_keep, theta, stage_row);
+    const int m = s.max_seqlen;
+    if (m <= 2048) launch_theta<256, 8>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 4096) launch_theta<256, 16>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 8192) launch_theta<256, 32>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 16384) launch_theta<512, 32>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 32768) launch_theta<1024, 32>(s, scores, sig_keep, theta, blocks, stream);
+    else {
+      const size_t row_bytes = (size_t)m * sizeof(uint32_t);
+      const int stage_row = row_bytes <= 200 * 1024;
+      const size_t dyn = stage_row ? row_bytes : 0;
+      if (dyn > 40 * 1024 &&
+          cudaFuncSetAttribute(theta_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+        return KVCRUSH_ERR_CUDA;
+      theta_stream_kernel<<<blocks, kSelectThreads, dyn, stream>>>(s, scores, sig_keep, theta, stage_row);
+    }
     if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
     th = theta;
   }
-  const long long n = (long long)s.n_layers * s.T;
-  binarise_pack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, scores, th, sigs);
+  const dim3 grid((unsigned)((s.T + 255) / 256), (unsigned)s.n_layers);
+  if (importance)
+    signature_pack_kernel<true><<<grid, 256, 0, stream>>>(s, scores, th, sigs, importance);
+  else
+    signature_pack_kernel<false><<<grid, 256, 0, stream>>>(s, scores, th, sigs, nullptr);
   return check_launch();
 }
 
@@ -196,6 +334,6 @@ extern "C" int kvcrush_signature_static(const kvcrush_problem_t* problem, const 
   float* theta = nullptr;
   const int prc = kvc::static_theta_ptr(&theta);
   if (prc != KVCRUSH_OK) return prc;
-  return kvc::launch_signature(s, scores_dev, sig_keep_dev, nullptr, sigs_dev, theta,
+  return kvc::launch_signature(s, scores_dev, sig_keep_dev, nullptr, sigs_dev, theta, nullptr,
                                static_cast<cudaStream_t>(stream));
 }

@@ -13,7 +13,9 @@
 namespace kvc {
 namespace tc {
 
-constexpr uint32_t kSpinLimit = 1u << 20;        // polls of one bounded barrier wait
+constexpr uint32_t kWaitPolls = 1u << 20;        // polls of one bounded barrier wait
+constexpr uint32_t kShortWaitPolls = 1u << 12;   // the same in the diagnostic build of the kernels (waits made to run out)
+constexpr uint32_t kDrainPolls = 1u << 20;       // polls granted to copies and MMAs in flight after a role gave up; never shortened
 
 // ------------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -38,9 +40,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when the wait ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+// Bounded wait of at most `polls` polls.  Returns false when the wait ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t polls) {
+  for (uint32_t i = 0; i < polls; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 31u) == 31u && *abort_flag) return false;
   }
@@ -446,12 +448,22 @@ inline EncodeTiledFn encode_fn() {
 }
 
 // 4-D view (channel, token, head, layer) of a token-major bf16 or fp16 tensor; box = 64 channels x 128 tokens.
+// A stride only matters along an axis longer than 1; there it must be positive (the TMA unit cannot repeat a row)
+// and inside the tensor map's 40-bit byte range.  Returns false for anything the map cannot describe.
 inline bool make_map(CUtensorMap* map, const TensorView& t, int D, int T, int H, int n_layers) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
   const cuuint64_t gdim[4] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)H, (cuuint64_t)n_layers};
-  auto stride_bytes = [](long long st) { return (cuuint64_t)(st > 0 ? st * 2 : 16); };
-  const cuuint64_t gstride[3] = {stride_bytes(t.st), stride_bytes(t.sh), stride_bytes(t.sl)};
+  const long long st[3] = {t.st, t.sh, t.sl};
+  cuuint64_t gstride[3];
+  for (int i = 0; i < 3; ++i) {
+    if (gdim[i + 1] > 1) {
+      if (st[i] <= 0 || st[i] >= (1LL << 38)) return false;
+      gstride[i] = (cuuint64_t)st[i] * 2;
+    } else {
+      gstride[i] = 16;                                // never used to step: any legal value
+    }
+  }
   const cuuint32_t box[4] = {64, 128u, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return enc(map, t.dtype == KVCRUSH_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(t.ptr), gdim, gstride, box, estr,

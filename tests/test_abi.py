@@ -80,22 +80,27 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
     assert lib.kvcrush_score(r(p), r(t), r(t), None, 0x100, None, 0, 0, None, 0, 0x100, None) == B.ERR_WORKSPACE
     assert lib.kvcrush_score(r(p), r(t), r(t), None, 0x100, None, 0, 7, 0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
     # signature: needs a rank or explicit thresholds; needs workspace when theta_out is NULL
-    assert lib.kvcrush_signature(r(p), 0x100, None, None, 0x100, None, None, 0, 0x100, None) == B.ERR_INVALID_ARG
-    assert lib.kvcrush_signature(r(p), 0x100, 0x100, None, 0x100, None, None, 0, 0x100, None) == B.ERR_WORKSPACE
+    assert lib.kvcrush_signature(r(p), 0x100, None, None, 0x100, None, None, None, 0, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_signature(r(p), 0x100, 0x100, None, 0x100, None, None, None, 0, 0x100, None) == B.ERR_WORKSPACE
     # select: anchor mode range, explicit anchor needs bits, workspace
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 5, None, 0, 0, 0, 0x100, 0x100, None, 0x100, 1 << 20,
+    assert lib.kvcrush_select(r(p), 0x100, None, 0x100, 0x100, 0x100, 5, None, 0, 0, 0, 0x100, 0x100, None, None, 0x100, 1 << 20,
                               0x100, None) == B.ERR_INVALID_ARG
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, B.ANCHOR_EXPLICIT, None, 0, 0, 0, 0x100, 0x100, None,
-                              0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, 0, 0, 0x100, 0x100, None, 0x100, 16,
+    assert lib.kvcrush_select(r(p), 0x100, None, 0x100, 0x100, 0x100, B.ANCHOR_EXPLICIT, None, 0, 0, 0, 0x100, 0x100, None,
+                              None, 0x100, 1 << 20, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_select(r(p), 0x100, None, 0x100, 0x100, 0x100, 0, None, 0, 0, 0, 0x100, 0x100, None, None, 0x100, 16,
                               0x100, None) == B.ERR_WORKSPACE
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, 0, -1, 0x100, 0x100, None, 0x100, 1 << 20,
+    assert lib.kvcrush_select(r(p), 0x100, None, 0x100, 0x100, 0x100, 0, None, 0, 0, -1, 0x100, 0x100, None, None, 0x100, 1 << 20,
                               0x100, None) == B.ERR_INVALID_ARG
-    assert lib.kvcrush_select(r(p), 0x100, 0x100, 0x100, 0x100, 0, None, 0, -1, 0, 0x100, 0x100, None, 0x100, 1 << 20,
+    assert lib.kvcrush_select(r(p), 0x100, None, 0x100, 0x100, 0x100, 0, None, 0, -1, 0, 0x100, 0x100, None, None, 0x100, 1 << 20,
                               0x100, None) == B.ERR_INVALID_ARG
+    # neither scores nor a ready importance array; a misaligned importance array
+    assert lib.kvcrush_select(r(p), None, None, 0x100, 0x100, 0x100, 0, None, 0, 0, 0, 0x100, 0x100, None, None, 0x100,
+                              1 << 20, 0x100, None) == B.ERR_INVALID_ARG
+    assert lib.kvcrush_select(r(p), None, 0x104, 0x100, 0x100, 0x100, 0, None, 0, 0, 0, 0x100, 0x100, None, None, 0x100,
+                              1 << 20, 0x100, None) == B.ERR_MISALIGNED
     # page-granular select: page size, page vector too long, too many pages per sequence, workspace
-    sp = lambda ps, prob=p, ws=1 << 20, ki=0: lib.kvcrush_select_pages(r(prob), 0x100, 0x100, ps, 0x100, 0x100, 0, None, 0,
-                                                                       ki, 0, 0x100, 0x100, None, 0x100, ws, 0x100, None)
+    sp = lambda ps, prob=p, ws=1 << 20, ki=0: lib.kvcrush_select_pages(r(prob), 0x100, None, 0x100, ps, 0x100, 0x100, 0, None, 0,
+                                                                       ki, 0, 0x100, 0x100, None, None, 0x100, ws, 0x100, None)
     assert sp(0) == B.ERR_INVALID_ARG
     assert sp(8, ki=-1) == B.ERR_INVALID_ARG
     assert sp(256) == B.ERR_UNSUPPORTED
@@ -119,6 +124,35 @@ def test_entry_points_reject_bad_arguments_before_launch(lib):
     assert lib.kvcrush_compact(r(p), r(t), r(t), 0x100, 0x100, 10, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_compact(r(p), r(t), None, 0x100, 0x100, 10, r(f16), None, 0x100, None) == B.ERR_INVALID_ARG
     assert lib.kvcrush_compact(r(p), r(t), None, 0x100, 0x100, -1, r(t), None, 0x100, None) == B.ERR_INVALID_ARG
+
+
+def _no_cuda_device():
+    import torch
+    return not torch.cuda.is_available()
+
+
+@pytest.mark.skipif(not _no_cuda_device(), reason="uses made-up device pointers: only where nothing can be launched")
+def test_auto_does_not_drop_to_the_cuda_cores_when_the_driver_lacks_the_encoder(lib):
+    """A problem the tensor-core kernels are made for (bf16, head_dim 64) on a machine whose driver cannot encode
+    tensor maps (here: no driver at all): KVCRUSH_SCORE_AUTO and KVCRUSH_SCORE_TENSOR refuse with
+    KVCRUSH_ERR_UNSUPPORTED instead of running the far slower CUDA-core kernels unnoticed.  A problem that the
+    tensor-core kernels cannot take anyway (fp32, or a stride of 0 along the head axis) is not refused by AUTO for
+    that reason: it goes on to the CUDA-core launch, which fails here for lack of a device."""
+    p = _problem()
+    r = ctypes.byref
+    t = B.TensorStruct(0x10000, B.BF16, 0, 100 * 8 * 64, 8 * 64, 64)
+    call = lambda q, k, impl, lse=None, ws=1 << 20: lib.kvcrush_score(r(p), r(q), r(k), lse, 0x100, None, 0, impl, 0x100,
+                                                                      ws, 0x100, None)
+    assert call(t, t, B.SCORE_AUTO) == B.ERR_UNSUPPORTED
+    assert call(t, t, B.SCORE_TENSOR) == B.ERR_UNSUPPORTED
+    f32 = B.TensorStruct(0x10000, B.FP32, 0, 100 * 8 * 64, 8 * 64, 64)
+    assert call(f32, f32, B.SCORE_AUTO) == B.ERR_CUDA
+    assert call(t, t, B.SCORE_SIMT) == B.ERR_CUDA
+    # with the row log-sum-exp supplied the workspace only holds the work counters: 256 bytes are enough,
+    # fewer are not; without it the full size is required
+    assert call(t, t, B.SCORE_SIMT, lse=0x100, ws=256) == B.ERR_CUDA
+    assert call(t, t, B.SCORE_SIMT, lse=0x100, ws=128) == B.ERR_WORKSPACE
+    assert call(t, t, B.SCORE_SIMT, ws=256) == B.ERR_WORKSPACE
 
 
 def test_missing_library_fails_loudly(monkeypatch):

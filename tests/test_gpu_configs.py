@@ -2,8 +2,8 @@
 times (all layers in one call per stage).
 
 Small shapes (1, 2) are compared with the oracle element by element, end to end.  For the large
-shapes the oracle computes what it can in seconds - all heads of one layer, a few heads of other
-layers, the complete tail columns and sampled rows of very long sequences - and everything else is
+shapes the oracle computes what it can in a minute or two - all heads of one layer, a few heads of
+other layers (whole columns, at L = 32768 too), tail columns and sampled rows elsewhere - and everything else is
 checked through properties that hold at any size: column sums of a head total the number of
 queries, kept counts equal the budget, kept lists are strictly ascending, and the oracle's
 selection run on the GPU's own float32 scores reproduces the GPU's kept set bit for bit."""
@@ -15,6 +15,10 @@ from paper_2503_00022_b200 import inputs
 import kvc_testlib as TL
 
 pytestmark = pytest.mark.gpu
+
+# End to end, a GPU/oracle disagreement is excused only within this many score tolerances of the threshold it
+# crosses: both the value and the threshold move by at most one tolerance (see GpuPass.check_end_to_end).
+E2E_FACTOR = 2.0 * (1.0 + 2.0 * TL.SCORE_RTOL)
 
 
 @pytest.fixture(scope="module")
@@ -159,6 +163,17 @@ class GpuPass:
 
     # ---- end to end against the oracle's own scores (one layer, all heads) -------------------------
     def check_end_to_end(self, layer):
+        """The GPU's pass against the oracle run on the oracle's own float64 scores.
+
+        With tol(x) = atol + rtol*|x| the scores satisfy |s_g - s_o| <= tol(s_o).  x - tol(x) and x + tol(x) are
+        monotone in x, so a rank statistic (the k-th largest) of the GPU's values lies within tol of the oracle's:
+        |theta_g - theta_o| <= tol(theta_o), and the same for the importance cut with tol_I(x) = Hq*atol + rtol*x.
+        A signature bit can therefore differ only where |s_o - theta_o| <= tol(s_o) + tol(theta_o), and a token can
+        change sides of the importance cut only where |I_o - cut_o| <= tol_I(I_o) + tol_I(cut_o): at most
+        E2E_FACTOR = 2*(1 + 2*rtol) times the tolerance at the threshold itself.  Every difference found is checked
+        against that bound, the largest observed ratio is returned, and where nothing differs the kept set must equal
+        the oracle's.  What the differences then do to the buckets is covered by check_selection_consistency on the
+        same layer (the oracle's steps on the GPU's scores reproduce the GPU's kept set bit for bit)."""
         w, cp = self.w, self.cp
         cu = w.cu_seqlens
         li = self.host[layer]
@@ -168,17 +183,19 @@ class GpuPass:
         o32 = O.to_scores32(c)
         ref = TL.oracle_select_layer(w, o32, self.b_imp, self.b_rep)
         sigs = cp.sigs.cpu().numpy().view(np.uint32)
-        exact = 0
+        out = dict(exact=0, bit_diffs=0, imp_diffs=0, max_bit_ratio=0.0, max_imp_ratio=0.0, sequences=w.n_seqs)
         for s, L in enumerate(w.seqlens):
             a, b = int(cu[s]), int(cu[s + 1])
             Hq = w.n_q_heads
-            # (ii) signature bits may differ only where the oracle score is within tolerance of theta_h
+            # (ii) signature bits may differ only where the oracle score is near theta_h
             gb = O.unpack_bits(sigs[layer, a:b], Hq)
             ob = O.unpack_bits(ref[s]["sig"], Hq)
             th = ref[s]["theta"].astype(np.float64)
             for t, h in np.argwhere(gb != ob):
-                # |s_o - theta_o| <= |s_o - s_g| + |theta_g - theta_o|: twice the score tolerance (plus slack)
-                assert abs(float(o32[h, a + t]) - th[h]) <= 2.5 * (TL.SCORE_ATOL + TL.SCORE_RTOL * abs(th[h])), (s, t, h)
+                ratio = abs(float(o32[h, a + t]) - th[h]) / (TL.SCORE_ATOL + TL.SCORE_RTOL * abs(th[h]))
+                assert ratio <= E2E_FACTOR, (s, t, h, ratio)
+                out["max_bit_ratio"] = max(out["max_bit_ratio"], ratio)
+                out["bit_diffs"] += 1
             # (i) important sets may differ only for tokens whose oracle importance is near the cut
             I_o = O.importance(np.ascontiguousarray(o32[:, a:b]), w.n_kv_heads)
             bi = int(self.b_imp[s])
@@ -188,12 +205,16 @@ class GpuPass:
             if bi > 0 and bi < L:
                 cut = np.sort(I_o)[::-1][bi - 1]
                 for t in imp_o ^ imp_g:
-                    assert abs(I_o[t] - cut) <= 2.5 * (Hq * TL.SCORE_ATOL + TL.SCORE_RTOL * cut), (s, t)
+                    ratio = abs(I_o[t] - cut) / (Hq * TL.SCORE_ATOL + TL.SCORE_RTOL * cut)
+                    assert ratio <= E2E_FACTOR, (s, t, ratio)
+                    out["max_imp_ratio"] = max(out["max_imp_ratio"], ratio)
+                    out["imp_diffs"] += 1
             same_inputs = np.array_equal(gb, ob) and imp_o == imp_g
             if same_inputs:                      # (iv) then the kept set and the reduced cache match exactly
                 np.testing.assert_array_equal(cp.kept(layer, s), ref[s]["idx"].astype(np.int32))
-                exact += 1
-        return exact
+                out["exact"] += 1
+        print("end to end %s layer %d: %s" % (w.name, layer, out))
+        return out
 
 
 def test_cfg1_small_fp32_end_to_end(B):
@@ -231,10 +252,12 @@ def test_cfg4_llama3_gqa_32k_full_size(B):
     gp.check_invariants()
     gp.check_selection_consistency([0, 9, 31])
     gp.check_compaction([31])
+    # layer 0: complete columns (all 32768 queries of the oracle, a minute or two on the host cores) and every
+    # row's log-sum-exp for the whole first KV group and four heads of other groups
+    gp.check_scores_heads(0, [0, 1, 2, 3, 4, 13, 22, 31])
     heads = [0, 3, 4, 31]                                    # two heads of one KV group, two others
-    gp.check_scores_tail(0, heads, 0, 768)
-    gp.check_scores_tail(31, heads, 0, 300)
-    gp.check_lse_rows(0, heads, 0, [0, 127, 128, 5000, 16383, 30000])
+    gp.check_scores_tail(31, heads, 0, 768)
+    gp.check_lse_rows(31, heads, 0, [0, 127, 128, 5000, 16383, 30000])
 
 
 def test_cfg5_ragged_batch16_full_size(B):

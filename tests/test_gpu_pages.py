@@ -31,6 +31,9 @@ def _run_pages(B, scores, Hkv, seqlens, P, b_imp, b_rep, mode=0, explicit=None, 
     cp.select(ds)
     torch.cuda.synchronize()
     cp.check_status()
+    pages = (np.asarray(seqlens, dtype=np.int64) + P - 1) // P
+    want = np.minimum(np.broadcast_to(np.asarray(b_imp, dtype=np.int64) + np.asarray(b_rep), (n_layers, len(seqlens))), pages[None])
+    np.testing.assert_array_equal(cp.n_kept.cpu().numpy(), want)         # the optional per-segment count output
     return cp
 
 

@@ -27,7 +27,7 @@ def _dev():
 # signature + select on oracle scores
 # ---------------------------------------------------------------------------------------------
 
-def _select_case(B, Hq, Hkv, seqlens, budgets, n_layers, ties, mode, seed, sig_keep=None):
+def _select_case(B, Hq, Hkv, seqlens, budgets, n_layers, ties, mode, seed, sig_keep=None, share_importance=True):
     import torch
     dev = _dev()
     S, T = len(seqlens), int(sum(seqlens))
@@ -41,8 +41,11 @@ def _select_case(B, Hq, Hkv, seqlens, budgets, n_layers, ties, mode, seed, sig_k
     explicit = inputs.random_anchor_bits(Hq, seed + 5)
     w = inputs.Workload("t", n_layers, Hq, Hkv, 16, tuple(seqlens), inputs.FP32, inputs.FP32, 0.25)
     prob = B.Problem(n_layers, Hq, Hkv, 16, seqlens, device=dev)
+    # share_importance: the signature stage writes the token importance and the selection stage takes it over;
+    # without it the selection stage makes its own pass over the scores
     cp = B.CompressionPass(prob, b_imp[None, :], b_rep[None, :], sig_keep=sig_keep, anchor_mode=mode,
-                           anchor_bits=explicit if mode == B.ANCHOR_EXPLICIT else None)
+                           anchor_bits=explicit if mode == B.ANCHOR_EXPLICIT else None,
+                           share_importance=share_importance)
     dscores = torch.from_numpy(scores).to(dev)
     for rep in range(2):                      # twice: results must not depend on leftover scratch
         cp.signature(dscores)
@@ -51,6 +54,8 @@ def _select_case(B, Hq, Hkv, seqlens, budgets, n_layers, ties, mode, seed, sig_k
         cp.check_status()
         sigs = cp.sigs.cpu().numpy().view(np.uint32)
         theta = cp.theta.cpu().numpy()
+        np.testing.assert_array_equal(cp.n_kept.cpu().numpy(),        # the optional per-segment count output
+                                      np.tile(np.minimum(b_imp + b_rep, np.asarray(seqlens)), (n_layers, 1)))
         for l in range(n_layers):
             ref = TL.oracle_select_layer(w, scores[l], b_imp, b_rep,
                                          None if sig_keep is None else np.asarray(sig_keep).reshape(-1),
@@ -82,6 +87,22 @@ def test_signature_and_select_bit_exact_on_oracle_scores(B, Hq, Hkv, seqlens, bu
 
 def test_select_long_sequence_32k(B):
     _select_case(B, 32, 8, [32768], [(3277, 3277)], 1, 0, 0, seed=9)
+    _select_case(B, 32, 8, [32768], [(3277, 3277)], 1, 0, 0, seed=9, share_importance=False)
+
+
+@pytest.mark.parametrize("Hq,Hkv,seqlens,budgets,ties,mode", [
+    (32, 8, [1000, 37, 2049], [(100, 150), (5, 4), (300, 212)], 0, 0),
+    (32, 8, [1000, 333], [(100, 150), (40, 43)], 4, 0),
+    (40, 10, [777, 1025], [(64, 32), (100, 101)], 2, 1),
+])
+def test_select_computes_the_importance_itself_when_none_is_handed_over(B, Hq, Hkv, seqlens, budgets, ties, mode):
+    _select_case(B, Hq, Hkv, seqlens, budgets, 2, ties, mode, seed=300 + Hq, share_importance=False)
+
+
+def test_signature_thresholds_for_rows_beyond_the_register_kernel(B):
+    """Rows longer than 32768 tokens take the streaming threshold kernel."""
+    _select_case(B, 4, 2, [40000, 70], [(500, 300), (7, 9)], 1, 0, 0, seed=17)
+    _select_case(B, 4, 2, [33000], [(100, 50)], 1, 3, 0, seed=18)
 
 
 def test_signature_rank_other_than_budget_and_explicit_theta(B):
@@ -171,11 +192,25 @@ def _score_case(B, w, impl, n_layers=None):
     torch.cuda.synchronize()
     assert status.cpu().tolist()[0] == 0, status.cpu().tolist()
     g, gl = scores.cpu().numpy(), lse.cpu().numpy()
+    oracle_c, oracle_lse = [], []
     for i, li in enumerate(lis):
         c, ol = TL.oracle_scores_layer(w, li)
         ok = TL.within_score_tolerance(g[i], c)
         assert ok.all(), (w.name, i, np.argwhere(~ok)[:5], g[i][~ok][:5], c[~ok][:5])
         np.testing.assert_allclose(gl[i], ol, rtol=0, atol=2e-4)
+        oracle_c.append(c)
+        oracle_lse.append(ol)
+    # the row log-sum-exp as a prefill kernel would hand it over - here the ORACLE's, rounded to float32, so that
+    # nothing of the library's first sweep is involved: the second sweep alone must reproduce the oracle's column sums
+    lse_o = torch.from_numpy(np.stack(oracle_lse).astype(np.float32)).to(dev)
+    scores3 = torch.full_like(scores, -1.0)
+    B.kvcrush_score(prob, dq, dk, scores3, lse_in=lse_o, impl=impl, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0
+    g3 = scores3.cpu().numpy()
+    for i, c in enumerate(oracle_c):
+        ok = TL.within_score_tolerance(g3[i], c)
+        assert ok.all(), (w.name, "oracle lse", i, np.argwhere(~ok)[:5], g3[i][~ok][:5], c[~ok][:5])
     # supplying the row log-sum-exp skips the first sweep and gives the same scores
     scores2 = torch.empty_like(scores)
     B.kvcrush_score(prob, dq, dk, scores2, lse_in=lse, impl=impl, workspace=ws, status=status)
@@ -301,6 +336,51 @@ def test_score_leaves_at_once_when_status_already_flags_an_error(B):
                     impl=B.SCORE_TENSOR, workspace=ws, status=status)
     torch.cuda.synchronize()
     assert status.cpu().tolist()[0] == 0 and bool((scores >= 0).all())
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable(B):
+    """Every barrier wait of the tensor-core kernels is bounded.  Here one is made to run out, on the smallest problem
+    there is (one work item, one thread block): through the library's diagnostic entry point (exported, not part of
+    the public header) the producer warp fetches its work item and then stops before announcing it and before issuing
+    any copy, and the kernels run in their instantiation with a short poll limit.  Nothing is in flight, so the
+    consumers' first waits expire, the block flags the status word, frees its tensor memory and the kernel returns
+    normally; the second sweep, enqueued by the same call, finds the status word set and leaves at once.  The outputs
+    stay untouched, and the same problem goes through the public entry point once the word is cleared."""
+    import ctypes
+    import torch
+    dev = _dev()
+    lib = B.lib()
+    fn = lib.kvcrush_diag_score
+    vp, i32 = ctypes.c_void_p, ctypes.c_int
+    fn.restype = i32
+    fn.argtypes = [ctypes.POINTER(B.ProblemStruct), ctypes.POINTER(B.TensorStruct), ctypes.POINTER(B.TensorStruct),
+                   vp, vp, vp, i32, i32, vp, ctypes.c_size_t, vp, vp, i32, i32]
+    w = inputs.Workload("one_item", 1, 1, 1, 128, (128,), inputs.BF16, inputs.BF16, 0.25, base_seed=55)
+    lis, q, k, _, _ = TL.stack_layers(w, range(1), with_cache=False)
+    prob = B.Problem(1, 1, 1, 128, w.seqlens, device=dev)
+    dq, dk = TL.torch_storage(q, w.qk_dtype, dev), TL.torch_storage(k, w.qk_dtype, dev)
+    qs, ks = B.tensor_struct(dq), B.tensor_struct(dk)
+    scores = torch.full((1, 1, 128), -5.0, dtype=torch.float32, device=dev)
+    lse = torch.full((1, 1, 128), -7.0, dtype=torch.float32, device=dev)
+    ws = torch.empty(B.kvcrush_workspace_size(prob, B.STAGE_SCORE), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    stream = int(torch.cuda.current_stream().cuda_stream)
+    rc = fn(prob.ref, ctypes.byref(qs), ctypes.byref(ks), None, scores.data_ptr(), lse.data_ptr(), 0, B.SCORE_TENSOR,
+            ws.data_ptr(), ws.numel(), status.data_ptr(), stream, 1, 1)
+    assert rc == B.OK
+    torch.cuda.synchronize()                                 # the kernels came back by themselves
+    st = status.cpu().tolist()
+    assert st[0] == B.DEV_TIMEOUT and st[1] == 1 and st[2] == 0, st          # kernel id 1: the row sweep; block 0
+    assert bool((scores == -5.0).all()) and bool((lse == -7.0).all())
+    # the public entry point gives the oracle's scores on the same context once the word is cleared
+    status.zero_()
+    scores.fill_(-5.0)
+    B.kvcrush_score(prob, dq, dk, scores, lse_out=lse, impl=B.SCORE_TENSOR, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0
+    c, ol = TL.oracle_scores_layer(w, lis[0])
+    assert TL.within_score_tolerance(scores.cpu().numpy()[0], c).all()
+    np.testing.assert_allclose(lse.cpu().numpy()[0], ol, rtol=0, atol=2e-4)
 
 
 def test_pass_replays_from_a_cuda_graph(B):
