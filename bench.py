@@ -34,7 +34,10 @@ from paper_2503_00022_b200 import inputs  # noqa: E402
 METRIC = "prompt tokens compressed/s (score+select+compact)"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg3_llama2_32l_8k"
-NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP = 138.2e6   # (276.0 + 276.7) MB / 2 sweeps / 2 layers: dram__bytes_read + dram__bytes_write
+# dram__bytes_read + dram__bytes_write of one sweep launch per layer, from the ncu capture of the 2-layer case:
+# (276.0 + 276.7) MB / 2 sweeps / 2 layers.  Valid for the kernel source named in NCU_TRAFFIC_SOURCE only.
+NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP = 138.2e6
+NCU_TRAFFIC_SOURCE = "ncu capture of score_persist_kernel at commit ec18db7 (2 layers of the workload, scaled by the layer count)"
 
 
 def measured_peaks():
@@ -176,71 +179,129 @@ def host_inputs(w: inputs.Workload, pinned: bool):
 # CPU oracle timing (cpu_baseline leg and --impl reference)
 # ---------------------------------------------------------------------------------------------
 
-def oracle_sample(w: inputs.Workload, max_heads=None):
-    """Times the float64 oracle on a bounded sample of the workload and scales to one step.
-
-    Sample: the score step for the first H_s query heads of layer 0 (H_s = host threads, at most
-    all heads) on the longest sequence, and signature + selection + compaction of layer 0's longest
-    sequence on seeded stand-in scores.  The step estimate scales the score time by
-    (layers * heads * causal entries) / sampled entries and the rest by layers * sequences-length share.
-    """
+def oracle_layer_pass(w: inputs.Workload, layer: int, n_heads: int = 0):
+    """One pass of the float64 oracle over one layer of the workload, timed: the score step for every sequence
+    (all query heads; the first ``n_heads`` only when 0 < n_heads < all), then thresholds, signatures, selection
+    and compaction of every sequence on the oracle's own float32 scores (on seeded stand-in scores when only
+    some heads were scored).  Returns (seconds, heads scored)."""
     from oracle import kvcrush_oracle as O
-    threads = O.n_threads()
-    s_long = int(np.argmax(w.seqlens))
-    L = w.seqlens[s_long]
-    cu = w.cu_seqlens
-    li = inputs.layer_inputs(w, 0)
-    hs = min(w.n_q_heads, max(1, threads if max_heads is None else max_heads))
+    hs = w.n_q_heads if not n_heads or n_heads >= w.n_q_heads else n_heads
     G = w.n_q_heads // w.n_kv_heads
-    hk = sorted(set(h // G for h in range(hs)))
-    a, b = int(cu[s_long]), int(cu[s_long + 1])
-    q = inputs.widen(li.q[a:b, :hs], w.qk_dtype)
-    # keep the GQA mapping of the sampled heads: expand their KV heads to one per query head
-    k = inputs.widen(li.k[a:b][:, [h // G for h in range(hs)]], w.qk_dtype)
-    del hk
-    t0 = time.perf_counter()
-    O.scores(q, k, w.causal)
-    t_score = time.perf_counter() - t0
-    entries_sample = hs * (L * (L + 1) // 2 if w.causal else L * L)
-    entries_step = w.n_layers * w.n_q_heads * sum(x * (x + 1) // 2 if w.causal else x * x for x in w.seqlens)
+    cu = w.cu_seqlens
+    li = inputs.layer_inputs(w, layer)
     b_imp, b_rep = w.budgets()
-    s32 = inputs.random_scores(w.n_q_heads, L, 7)
     t0 = time.perf_counter()
-    theta = O.thresholds(s32, int(b_imp[s_long] + b_rep[s_long]))
-    sig = O.signatures(s32, theta)
-    idx, _ = O.select(s32, sig, int(b_imp[s_long]), int(b_rep[s_long]), w.n_kv_heads)
-    O.compact(li.k_cache[a:b], idx)
-    O.compact(li.v_cache[a:b], idx)
-    t_rest = time.perf_counter() - t0
-    step_s = t_score * entries_step / entries_sample + t_rest * w.n_layers * w.total_tokens / L
-    desc = (f"score: layer 0, {hs} of {w.n_q_heads} heads, L={L} ({t_score:.2f} s); signature+select+compact: "
-            f"layer 0, L={L} on seeded stand-in scores ({t_rest:.2f} s); scaled to {w.n_layers} layers x "
-            f"{w.n_q_heads} heads x {w.total_tokens} tokens")
-    return dict(value=w.total_tokens / step_s, unit=UNIT, cores=threads, kind="oracle", sample=desc,
-                est_step_s=step_s)
+    for s in range(w.n_seqs):
+        a, b = int(cu[s]), int(cu[s + 1])
+        if hs == w.n_q_heads:
+            c, _ = O.scores(inputs.widen(li.q[a:b], w.qk_dtype), inputs.widen(li.k[a:b], w.qk_dtype), w.causal)
+            s32 = O.to_scores32(c)
+        else:
+            # the sampled heads keep their GQA mapping: their KV heads are expanded to one per query head
+            O.scores(inputs.widen(li.q[a:b, :hs], w.qk_dtype),
+                     inputs.widen(li.k[a:b][:, [h // G for h in range(hs)]], w.qk_dtype), w.causal)
+            s32 = inputs.random_scores(w.n_q_heads, b - a, 7 + s)
+        theta = O.thresholds(s32, int(b_imp[s] + b_rep[s]))
+        sig = O.signatures(s32, theta)
+        idx, _ = O.select(s32, sig, int(b_imp[s]), int(b_rep[s]), w.n_kv_heads)
+        O.compact(li.k_cache[a:b], idx)
+        O.compact(li.v_cache[a:b], idx)
+    return time.perf_counter() - t0, hs
+
+
+def oracle_sample_desc(w, hs, secs, layers):
+    what = "all %d heads" % w.n_q_heads if hs == w.n_q_heads else "%d of %d heads (selection on stand-in scores)" % (hs, w.n_q_heads)
+    return ("oracle pass (score, thresholds, signatures, selection, compaction) over layer(s) %s of %d, %s, "
+            "all %d sequence(s), %d tokens: %.2f s per layer; the step figure is that time x %d layers%s"
+            % (layers, w.n_layers, what, w.n_seqs, w.total_tokens, secs, w.n_layers,
+               "" if hs == w.n_q_heads else " x %d/%d heads for the score part" % (w.n_q_heads, hs)))
+
+
+def cpu_baseline_leg(w: inputs.Workload):
+    """The oracle as it stands on this machine's host cores: one whole layer of the workload, scaled by the layer
+    count (layers are independent and of equal size)."""
+    from oracle import kvcrush_oracle as O
+    O.build_c()
+    secs, hs = oracle_layer_pass(w, 0)
+    step_s = secs * w.n_layers
+    return dict(value=w.total_tokens / step_s, unit=UNIT, cores=O.n_threads(), kind="oracle",
+                sample=oracle_sample_desc(w, hs, secs, "0"), extrapolation_factor=w.n_layers, sample_s=secs)
+
+
+def workload_config(w: inputs.Workload, world: int, args, b_imp, b_rep):
+    """The `config` object: the same keys and values from both arms."""
+    eq, ec = inputs.storage_itemsize(w.qk_dtype), inputs.storage_itemsize(w.cache_dtype)
+    row = w.n_layers * w.total_tokens * w.head_dim
+    # Q and K for scoring, the K/V cache to compact (K serves as its own cache when the types agree)
+    resident_bytes = row * (w.n_q_heads + w.n_kv_heads) * eq + row * w.n_kv_heads * ec * (1 if w.cache_dtype == w.qk_dtype else 2)
+    return {"workload": w.name, "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
+            "head_dim": w.head_dim, "n_seqs": w.n_seqs, "total_tokens": w.total_tokens,
+            "budget_per_seq": [int(b_imp[0] + b_rep[0])], "cache_dtype": w.cache_dtype,
+            "l2": "inputs %s L2 (%.2f GiB resident per step)" % ("larger than" if resident_bytes > 126e6 else "smaller than", resident_bytes / 2 ** 30),
+            "parallelism": "replicas only" if world > 1 else "single GPU",
+            "query_window": args.window, "pool_kernel": args.pool, "page_size": args.page_size,
+            "keep_initial": args.keep_initial, "keep_recent": max(args.window, args.keep_recent)}
+
+
+REFERENCE_BUDGET_S = 450.0     # the whole --impl reference run (warm-up + steps) is sized to end within this
 
 
 def run_reference(args, w):
-    rank, _, _ = dist_env()
+    """The oracle, as it stands, on the host cores.  One step = the oracle's whole pass over ONE layer of the
+    workload (step i takes layer i mod layers); `ms_per_step` is the measured time of such a step and `value`
+    divides the workload's tokens by that time x the layer count (`extrapolation_factor`).  With --steps equal to
+    the layer count and --warmup 0 every layer is visited once and `full_pass_s` is the whole workload, measured."""
+    rank, world, _ = dist_env()
     if rank != 0:                      # under torchrun only rank 0 runs the CPU oracle; the others leave
         return
     from oracle import kvcrush_oracle as O
     O.build_c()
-    for _ in range(max(0, min(args.warmup, 1))):
-        oracle_sample(w, max_heads=2)
-    vals = [oracle_sample(w) for _ in range(max(1, min(args.steps, 3)))]
-    best = max(vals, key=lambda v: v["value"])
-    value = float(np.mean([v["value"] for v in vals]))
+    threads = O.n_threads()
+    b_imp, b_rep = w.budgets()
+    t_run = time.perf_counter()
+    # calibration (not a step): one round of heads on layer 0 tells whether whole layers fit the time budget
+    cal_heads = min(w.n_q_heads, threads)
+    cal_s, _ = oracle_layer_pass(w, 0, cal_heads)
+    rounds = -(-w.n_q_heads // cal_heads)
+    n_req = args.warmup + args.steps
+    heads = 0                                              # whole layers
+    steps, warmup = args.steps, args.warmup
+    if cal_s * rounds * n_req > REFERENCE_BUDGET_S:
+        heads = cal_heads if cal_heads < w.n_q_heads else 0
+        per = cal_s if heads else cal_s * rounds
+        fit = max(1, int(REFERENCE_BUDGET_S / per))
+        if fit < n_req:                                    # still too long: fewer steps, said in the line
+            warmup = min(warmup, max(0, fit - 1) // 4)
+            steps = max(1, min(steps, fit - warmup))
+    for i in range(warmup):
+        oracle_layer_pass(w, i % w.n_layers, heads)
+    secs, layers, hs = [], [], w.n_q_heads
+    for i in range(steps):
+        layer = (warmup + i) % w.n_layers
+        t, hs = oracle_layer_pass(w, layer, heads)
+        secs.append(t)
+        layers.append(layer)
+    mean_s = float(np.mean(secs))
+    factor = w.n_layers * (w.n_q_heads / hs)
+    step_s = mean_s * factor
+    value = w.total_tokens / step_s
+    sample = oracle_sample_desc(w, hs, mean_s, "%d..%d" % (layers[0], layers[-1]) if len(set(layers)) > 1 else str(layers[0]))
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * w.total_tokens / value, "higher_is_better": True,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": 1e3 * mean_s, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
-                   "head_dim": w.head_dim, "seqlens": list(w.seqlens)[:4], "note": "each step is a bounded sample scaled to the workload"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": best["cores"], "kind": "oracle", "sample": best["sample"]},
+        "config": workload_config(w, world, args, b_imp, b_rep),
+        "extrapolation_factor": factor, "workload_ms_per_step": 1e3 * step_s,
+        "steps_requested": args.steps, "warmup_requested": args.warmup,
+        "note": "a step is the oracle's pass over one layer (measured); value = workload tokens / (ms_per_step x extrapolation_factor)",
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "gpu_launches": 0,
+        "gpu_launches": 0, "run_s": None,
     }
+    if hs == w.n_q_heads and sorted(set(layers)) == list(range(w.n_layers)):
+        line["full_pass_s"] = float(np.sum([np.mean([t for t, l in zip(secs, layers) if l == x]) for x in range(w.n_layers)]))
+        line["full_pass_tokens_per_s"] = w.total_tokens / line["full_pass_s"]
+    line["run_s"] = time.perf_counter() - t_run
     print(json.dumps(line))
 
 
@@ -326,6 +387,36 @@ def run_ours(args, w):
     stage_ms = stage_all.mean(axis=0)
     total_ms = max_over_ranks(total_ms, dev, world)
     ms_per_step = total_ms / args.steps
+
+    # ---- the unchanged pass looped for several seconds: the board settles at its power limit and the SM clock it
+    # sustains there, which is the condition the sustained GEMM peak was measured under ----
+    sus = None
+    if args.sustained_s > 0:
+        n_sus = max(args.steps, int(np.ceil(args.sustained_s * 1e3 / ms_per_step)))
+        ev_s = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n_sus)]
+        sampler_s = ClockSampler(local) if rank == 0 else None
+        barrier()
+        t_b = time.time()
+        e0.record()
+        for i in range(n_sus):
+            ev_s[i][0].record()
+            cp.score(q, k)
+            if cp.pooled is not None:
+                cp.pool()
+            ev_s[i][1].record()
+            cp.signature()
+            cp.select()
+            cp.compact(kc, vc)
+        e1.record()
+        barrier()
+        t_e = time.time()
+        clocks_s = sampler_s.stop(t_b + 1.0, t_e) if sampler_s else None      # the first second is the ramp
+        cp.check_status()
+        sus_ms = max_over_ranks(e0.elapsed_time(e1), dev, world) / n_sus
+        half = n_sus // 2                                                     # settled part of the loop
+        sus_score_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in ev_s[half:]]))
+        sus = dict(steps=n_sus, seconds=sus_ms * n_sus * 1e-3, ms_per_step=sus_ms, score_ms_settled=sus_score_ms,
+                   clocks=clocks_s)
 
     # ---- the same pass when the caller already has the row log-sum-exp (a prefill attention kernel returns it):
     # the first sweep is skipped.  Reported beside the headline, never instead of it.
@@ -460,18 +551,40 @@ def run_ours(args, w):
         eb = inputs.storage_itemsize(w.cache_dtype)
         work["compact_bytes"] = 2 * 2 * cp.total_kept * args.page_size * w.n_kv_heads * w.head_dim * eb
     score_s = stage_ms[0] * 1e-3
-    tensor_path = B.lib() is not None and w.qk_dtype == inputs.BF16 and w.head_dim in (64, 128)
-    achieved_tf = work["score_flops"] / score_s / 1e12
-    peak_tf = peaks["bf16_tflops_sustained"]
-    # dram__bytes_read + dram__bytes_write of one sweep launch: 138 MB per layer in the ncu capture of a 2-layer case
-    # of this workload (profiles/score_persist_kernel_cfg3_2layers.md); proportional to the layer count
-    traffic = NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP * w.n_layers if (tensor_path and w.name.startswith(DEFAULT_WORKLOAD) and not args.window) else None
-    roofline = {"bound": "tensor" if tensor_path else "alu", "kernel": "score_persist_kernel (two sweep launches per step; per-launch figures)" if tensor_path else "score SIMT",
-                "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
-                "traffic": traffic, "algorithmic_flops_per_launch": work["score_flops"] / 2,
-                "launch_ms": float(stage_ms[0]) / 2, "peak_source": peaks["source"] + " (sustained bf16)",
-                "frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved_tf / 2250.0,
-                "exps_per_s": work["exps"] / score_s}
+    tensor_path = cp.impl != B.SCORE_SIMT and w.qk_dtype in (inputs.BF16, inputs.FP16) and w.head_dim % 8 == 0 and w.head_dim <= 128
+    short_tf = work["score_flops"] / score_s / 1e12
+    if tensor_path:
+        # Headline fraction: the score stage inside the seconds-long loop against the sustained GEMM peak (both at the
+        # board's power limit); beside it the K-step loop against the burst peak (both short).
+        sus_tf = work["score_flops"] / (sus["score_ms_settled"] * 1e-3) / 1e12 if sus else short_tf
+        launch_ms = (sus["score_ms_settled"] if sus else float(stage_ms[0])) / 2
+        whole = w.name == DEFAULT_WORKLOAD or w.name.startswith(DEFAULT_WORKLOAD + "_")
+        traffic = NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP * w.n_layers if (whole and not args.window) else None
+        roofline = {"bound": "tensor", "kernel": "score_persist_kernel (two sweep launches per step; per-launch figures)",
+                    "achieved": sus_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": sus_tf / peaks["bf16_tflops_sustained"],
+                    "timing": ("score stage, CUDA events, settled half of a %.1f s loop of the whole pass" % sus["seconds"]) if sus else "score stage of the timed steps",
+                    "peak_source": peaks["source"] + " (sustained bf16: seconds-long loop under the power cap)",
+                    "traffic": traffic, "traffic_source": NCU_TRAFFIC_SOURCE if traffic else None,
+                    "algorithmic_flops_per_launch": work["score_flops"] / 2, "launch_ms": launch_ms,
+                    "short_loop": {"achieved": short_tf, "peak": peaks["bf16_tflops"], "frac": short_tf / peaks["bf16_tflops"],
+                                   "launch_ms": float(stage_ms[0]) / 2,
+                                   "note": "score stage of the %d timed steps against the burst bf16 peak" % args.steps},
+                    "frac_of_nominal_2250": sus_tf / 2250.0,
+                    "exps_per_s": work["exps"] / (2 * launch_ms * 1e-3)}
+        if sus and sus["clocks"]:
+            ghz = sus["clocks"]["sm_mhz"] * 1e-3
+            roofline["sm_ghz_sustained"] = ghz
+            roofline["launch_ms_x_ghz"] = launch_ms * ghz          # clock-independent cost of one sweep: Mcycles
+    else:
+        # fp32 FMA on the CUDA cores: 128 lanes x 2 flop per SM per clock at the SM clock sampled during the timed steps
+        n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+        mhz = clocks["sm_mhz"] if clocks else 1965.0
+        peak_tf = n_sm * 128 * 2 * mhz * 1e6 / 1e12
+        roofline = {"bound": "alu", "kernel": "score SIMT kernels (fp32 FMA on the CUDA cores)", "achieved": short_tf,
+                    "peak": peak_tf, "unit": "TFLOP/s", "frac": short_tf / peak_tf, "traffic": None,
+                    "peak_source": "derived: %d SMs x 128 fp32 lanes x 2 flop x %.0f MHz (sampled SM clock)" % (n_sm, mhz),
+                    "algorithmic_flops_per_launch": work["score_flops"] / 2, "launch_ms": float(stage_ms[0]) / 2}
     hbm = peaks["hbm_gbs"]
     stages = {
         "score_ms": float(stage_ms[0]), "signature_ms": float(stage_ms[1]), "select_ms": float(stage_ms[2]),
@@ -489,23 +602,17 @@ def run_ours(args, w):
     }
     cpu = None
     if not args.no_cpu_baseline:
-        from oracle import kvcrush_oracle as O
-        O.build_c()
-        cpu = oracle_sample(w)
-        cpu.pop("est_step_s", None)
+        cpu = cpu_baseline_leg(w)
 
     tokens = w.total_tokens * world
+    # kernels of this library per step: two score sweeps, threshold select + signature pack (which also writes the token
+    # importance), the segment selection, the gather (+ pooling)
+    launches_per_step = 2 + 2 + (1 if cp.importance is not None else 2) + 1 + (1 if cp.pooled is not None else 0)
     line = {
         "metric": METRIC, "value": whole_job_value(w.total_tokens, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if w.qk_dtype == inputs.BF16 else "f32", "data": "synthetic",
-        "config": {"workload": w.name, "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
-                   "head_dim": w.head_dim, "n_seqs": w.n_seqs, "total_tokens": w.total_tokens,
-                   "budget_per_seq": [int(b_imp[0] + b_rep[0])], "cache_dtype": w.cache_dtype,
-                   "l2": "inputs larger than L2 (%.1f GiB resident per step)" % (h2d / 2 ** 30),
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "query_window": args.window, "pool_kernel": args.pool, "page_size": args.page_size,
-                   "keep_initial": args.keep_initial, "keep_recent": max(args.window, args.keep_recent)},
+        "config": workload_config(w, world, args, b_imp, b_rep),
         "layer_tokens_per_s": tokens * w.n_layers / (ms_per_step * 1e-3),
         "roofline": roofline, "stages": stages, "cpu_baseline": cpu,
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -513,7 +620,9 @@ def run_ours(args, w):
                 "overlap": "H2D, compute and D2H of consecutive layer chunks on three streams"},
         "lse_supplied": {"ms_per_step": lse_ms, "value": whole_job_value(w.total_tokens, world, lse_ms), "unit": UNIT,
                          "note": "row log-sum-exp given by the caller: one score sweep instead of two"},
-        "gpu_launches": (7 + (1 if cp.pooled is not None else 0)) * args.steps,
+        "sustained": sus,
+        "gpu_launches": launches_per_step * args.steps,
+        "gpu_launches_per_step": launches_per_step,
         "clocks": clocks,
     }
     print(json.dumps(line))
@@ -530,6 +639,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--layers", type=int, default=0, help="run only this many layers of the workload (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustained-s", type=float, default=4.0,
+                    help="also loop the pass for at least this many seconds (0 = skip); the roofline fraction is taken there")
     ap.add_argument("--window", type=int, default=0,
                     help="SnapKV-style importance: only the last WINDOW queries vote and those tokens are kept (0 = H2O, all queries)")
     ap.add_argument("--pool", type=int, default=0, help="max-pool the per-head scores with this odd kernel width (0 = off)")
