@@ -37,6 +37,13 @@ __device__ __forceinline__ unsigned long long importance_key(double v, int t, in
   return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
 }
 
+// floor(b * N / R) for N = q_nr * R + r_nr, 0 <= b <= R < 2^18: b * q_nr + floor(b * r_nr / R), in 32 bits when it fits.
+__device__ __forceinline__ int bucket_lo(int b, int q_nr, int r_nr, int R) {
+  const unsigned long long p = (unsigned long long)(unsigned)b * (unsigned)r_nr;
+  const unsigned frac = R < 65536 ? (unsigned)p / (unsigned)R : (unsigned)(p / (unsigned)R);
+  return b * q_nr + (int)frac;
+}
+
 __global__ void __launch_bounds__(256)
 importance_kernel(Shape s, const float* __restrict__ scores, int keep_initial, int keep_recent,
                   unsigned long long* __restrict__ keys) {
@@ -257,10 +264,44 @@ select_segment_kernel(Shape s, SelectArgs a) {
     }
     __syncthreads();
 
-    // one representative per equal-frequency bucket (one warp per bucket)
-    // bucket i covers sorted positions [floor(i*N/R), floor((i+1)*N/R)).  64-bit divisions are slow, so each
+    // one representative per equal-frequency bucket
+    // bucket i covers sorted positions [floor(i*N/R), floor((i+1)*N/R)); N = q_nr*R + r_nr
+    const int q_nr = N / b_rep, r_nr = N - q_nr * b_rep;
+    const int m_max = q_nr + (r_nr > 0 ? 1 : 0);                               // largest bucket
+    if (m_max <= 16) {
+      // Small buckets (the usual case: N/R is the compression ratio): 32 / gw buckets share a warp, gw = the power
+      // of two that holds a bucket, one lane per member.  sum_{h set in t} n_h = sum over members u of
+      // popc(sig_t & sig_u), so cost(t) = m * popc(sig_t) - 2 * sum_u popc(sig_t & sig_u): m_max shuffles inside
+      // the lane group.  |cost| <= 16 * 128 and t < 2^18, so (cost, t) packs into 31 bits and one warp-level
+      // minimum per lane group picks the representative, ties to the lower token.
+      int gw = 2;
+      while (gw < m_max) gw <<= 1;
+      const int per_warp = 32 / gw, sub = lane / gw, j = lane - sub * gw;
+      const unsigned gmask = (0xFFFFFFFFu >> (32 - gw)) << (sub * gw);
+      for (int b0 = warp * per_warp; b0 < b_rep; b0 += kWarps * per_warp) {
+        const int bkt = b0 + sub;
+        const bool live = bkt < b_rep;
+        const int lo = live ? bucket_lo(bkt, q_nr, r_nr, b_rep) : 0;
+        const int m = live ? bucket_lo(bkt + 1, q_nr, r_nr, b_rep) - lo : 0;
+        const bool member = j < m;
+        const int t = member ? sorted[lo + j] : 0;
+        uint32_t mine[4] = {0u, 0u, 0u, 0u};
+        _Pragma("unroll") for (int w = 0; w < W; ++w) mine[w] = member ? sig[(size_t)t * W + w] & head_mask(s.Hq, w) : 0u;
+        int ones = 0, shared = 0;
+        _Pragma("unroll") for (int w = 0; w < W; ++w) ones += __popc(mine[w]);
+        for (int u = 0; u < m_max; ++u)            // lanes past a bucket's last member hold zeros and add nothing
+          _Pragma("unroll") for (int w = 0; w < W; ++w) shared += __popc(mine[w] & __shfl_sync(kFull, mine[w], u, gw));
+        const int cost = m * ones - 2 * shared;
+        const uint32_t key = member ? ((uint32_t)(cost + 4096) << 18) | (uint32_t)t : 0xFFFFFFFFu;
+        const uint32_t best = __reduce_min_sync(gmask, key);
+        if (j == 0 && live) {
+          const uint32_t bt = best & 0x3FFFFu;
+          atomicOr(&rep_mask[bt >> 5], 1u << (bt & 31));
+        }
+      }
+    } else {
+    // Larger buckets: one warp per bucket.  64-bit divisions are slow, so each
     // warp divides once and then steps exactly: i*N = pos*R + rem, and the stride kWarps*N = step_q*R + step_r.
-    const int q_nr = N / b_rep, r_nr = N - q_nr * b_rep;                       // N = q_nr*R + r_nr
     const long long stride = (long long)kWarps * N;
     const int step_q = (int)(stride / b_rep), step_r = (int)(stride - (long long)step_q * b_rep);
     int pos = (int)(((long long)warp * N) / b_rep);
@@ -329,6 +370,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
         const uint32_t t = (uint32_t)best;
         atomicOr(&rep_mask[t >> 5], 1u << (t & 31));
       }
+    }
     }
     __syncthreads();
   }

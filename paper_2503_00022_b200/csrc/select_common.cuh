@@ -16,7 +16,7 @@ constexpr int kBins = 1 << kDigitBits;
 constexpr int kSmallList = 32;                 // candidates one warp ranks directly
 
 struct Scratch {
-  uint32_t hist[kBins];
+  alignas(16) uint32_t hist[kBins];
   unsigned long long red[2][kWarps];           // per-warp minimum / maximum
   unsigned long long small[kSmallList];
   unsigned long long sel_x;                    // result of a search step
@@ -50,8 +50,15 @@ __device__ __forceinline__ void find_digit_desc(const uint32_t* hist, int n_bins
   const int per = n_bins >= kT ? n_bins / kT : 1;           // bins per thread, walked from the top digit down
   const int n_act = n_bins / per;
   uint32_t local = 0;
-  if (tid < n_act)
-    for (int j = 0; j < per; ++j) local += hist[n_bins - 1 - (tid * per + j)];
+  if (tid < n_act) {
+    const int first = n_bins - (tid + 1) * per;              // the thread's bins are [first, first + per)
+    if (per % 4 == 0) {                                      // 16-byte loads: consecutive threads, consecutive quads
+      const uint4* q = reinterpret_cast<const uint4*>(hist + first);
+      for (int j = 0; j < per / 4; ++j) { const uint4 v = q[j]; local += (v.x + v.y) + (v.z + v.w); }
+    } else {
+      for (int j = 0; j < per; ++j) local += hist[first + j];
+    }
+  }
   uint32_t incl = local;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
@@ -92,6 +99,19 @@ __device__ __forceinline__ unsigned long long warp_rank_select(unsigned long lon
   const int src = __ffs(who) - 1;                     // equal candidates all qualify: any of them
   k_out = k_rem - __shfl_sync(kFull, gt, src);
   return __shfl_sync(kFull, v, src);
+}
+
+// The same for 32-bit candidates (one shuffle per candidate instead of two).
+__device__ __forceinline__ uint32_t warp_rank_select32(uint32_t v, int n, uint32_t k_rem, int lane) {
+  uint32_t gt = 0, ge = 0;
+  for (int j = 0; j < n; ++j) {
+    const uint32_t o = __shfl_sync(kFull, v, j);
+    gt += o > v;
+    ge += o >= v;
+  }
+  const bool hit = lane < n && gt < k_rem && k_rem <= ge;
+  const unsigned who = __ballot_sync(kFull, hit);
+  return __shfl_sync(kFull, v, __ffs(who) - 1);
 }
 
 // Sets bit i of imp_mask for the k items with the largest keys[0..n); equal keys are admitted in ascending

@@ -7,11 +7,11 @@
 //                             last few candidates directly.  Usually one histogram pass.
 //   theta_stream_kernel       the same result for longer rows: MSB-first radix select (4 sweeps of 8 bits) that
 //                             re-reads the row from memory (or from a shared-memory copy) in every sweep.
-//   signature_pack_kernel     one thread per (layer, token): loads the token's score of every head (32 loads in
-//                             flight), compares with that head's threshold and packs the bits; from the same
-//                             loads it can add up the token's importance I(t) in float64, in the fixed order
-//                             stage 3 defines, which saves stage 3 its own pass over the scores.
-//                             Lanes are consecutive tokens, so every per-head load is a coalesced 128-byte row.
+//   signature_pack_kernel     one block per (layer, 128 tokens): stages the [heads][tokens] tile of scores in shared
+//                             memory with 16-byte row loads, then one thread per token compares its score of every
+//                             head with that head's threshold and packs the bits; from the same tile it can add up
+//                             the token's importance I(t) in float64, in the fixed order stage 3 defines, which
+//                             saves stage 3 its own pass over the scores.
 #include "select_common.cuh"
 
 namespace kvc {
@@ -19,6 +19,9 @@ namespace kvc {
 namespace {
 
 constexpr int kSelectThreads = 512;
+#ifndef KVC_THETA_T8K
+#define KVC_THETA_T8K 512                      // threads of theta_select_kernel for rows of 4097..8192 tokens
+#endif
 constexpr int kThetaBits = 12;                 // radix digit of theta_select_kernel
 constexpr int kThetaBins = 1 << kThetaBits;
 
@@ -36,10 +39,10 @@ template <int kT, int kItems>
 __global__ void __launch_bounds__(kT)
 theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __restrict__ sig_keep,
                     float* __restrict__ theta) {
-  __shared__ uint32_t hist[kThetaBins];
+  __shared__ alignas(16) uint32_t hist[kThetaBins];
   __shared__ uint32_t red[2][32];
   __shared__ uint32_t small[sel::kSmallList];
-  __shared__ uint32_t small_n, sel_x;
+  __shared__ uint32_t small_n;
   __shared__ uint32_t found[3];
   __shared__ int warp_tot[32];
 
@@ -70,45 +73,52 @@ theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __
   lo = __reduce_min_sync(sel::kFull, lo);
   hi = __reduce_max_sync(sel::kFull, hi);
   if (lane == 0) { red[0][warp] = lo; red[1][warp] = hi; }
+  for (int i = tid; i < kThetaBins; i += kT) hist[i] = 0;
+  if (tid == 0) small_n = 0;
   __syncthreads();
   lo = __reduce_min_sync(sel::kFull, lane < kT / 32 ? red[0][lane] : 0xFFFFFFFFu);
   hi = __reduce_max_sync(sel::kFull, lane < kT / 32 ? red[1][lane] : 0u);
   const uint32_t base = lo, range = hi - lo;
+  // From here on key[j] holds x = key - base; slots past the end of the row hold 0, the row's minimum: they add to
+  // the count of the lowest values only, which a rank counted from the top (keep < L) never reaches beyond the
+  // real minimum itself.
+#pragma unroll
+  for (int j = 0; j < kItems; ++j) key[j] = j * kT + tid < L ? key[j] - base : 0u;
 
-  // x = key - base has `rem` significant bits; `top` is the value of the bits of x above them chosen so far
+  // x has `rem` significant bits; `top` is the value of the bits of x above them chosen so far
   int rem = range ? 32 - __clz(range) : 0;
   uint32_t top = 0, k_rem = (uint32_t)keep;
+  bool first = true;
   while (rem > 0) {
     const int w = rem < kThetaBits ? rem : kThetaBits, shift = rem - w, n_bins = 1 << w;
-    for (int i = tid; i < n_bins; i += kT) hist[i] = 0;
-    if (tid == 0) small_n = 0;
-    __syncthreads();
+    if (first) {                                             // every x counts and has no bits above the digit
 #pragma unroll
-    for (int j = 0; j < kItems; ++j) {
-      const uint32_t x = key[j] - base;
-      if (j * kT + tid < L && ((x >> 1) >> (rem - 1)) == top) atomicAdd(&hist[(x >> shift) & (uint32_t)(n_bins - 1)], 1u);
+      for (int j = 0; j < kItems; ++j) atomicAdd(&hist[key[j] >> shift], 1u);
+    } else {
+      for (int i = tid; i < n_bins; i += kT) hist[i] = 0;
+      if (tid == 0) small_n = 0;
+      __syncthreads();
+#pragma unroll
+      for (int j = 0; j < kItems; ++j)
+        if (((key[j] >> 1) >> (rem - 1)) == top) atomicAdd(&hist[(key[j] >> shift) & (uint32_t)(n_bins - 1)], 1u);
     }
+    first = false;
     __syncthreads();
     sel::find_digit_desc<kT>(hist, n_bins, k_rem, warp_tot, found);
     top = (top << w) | found[0];
     k_rem = found[1];
     const uint32_t live = found[2];
     rem = shift;
-    if (rem > 0 && live <= (uint32_t)sel::kSmallList) {     // few candidates: one warp ranks their remaining bits
+    if (rem > 0 && live <= (uint32_t)sel::kSmallList) {     // few candidates: one warp ranks them and finishes
 #pragma unroll
-      for (int j = 0; j < kItems; ++j) {
-        const uint32_t x = key[j] - base;
-        if (j * kT + tid < L && ((x >> 1) >> (rem - 1)) == top) small[atomicAdd(&small_n, 1u)] = x;
-      }
+      for (int j = 0; j < kItems; ++j)
+        if ((key[j] >> rem) == top) small[atomicAdd(&small_n, 1u)] = key[j];
       __syncthreads();
       if (warp == 0) {
-        uint32_t k_out;
-        const unsigned long long v = sel::warp_rank_select(lane < (int)live ? small[lane] : 0u, (int)live, k_rem, lane, k_out);
-        if (lane == 0) sel_x = (uint32_t)v;
+        const uint32_t x = sel::warp_rank_select32(lane < (int)live ? small[lane] : 0u, (int)live, k_rem, lane);
+        if (lane == 0) *out = key_to_float(base + x);
       }
-      __syncthreads();
-      top = sel_x;
-      rem = 0;
+      return;
     }
     __syncthreads();                                         // hist and found are rewritten by the next step
   }
@@ -205,47 +215,57 @@ theta_stream_kernel(Shape s, const float* __restrict__ scores, const int32_t* __
 
 // kImportance: also write I(t) = sum of the token's per-head scores (float64; heads ascending inside each KV
 // group, then the group sums ascending: sequential IEEE additions, so the value is bit-reproducible).
-// Grid: (token blocks, layers).  The thresholds of the block's sequence sit in shared memory when all its tokens
-// belong to one sequence (always, with one sequence per batch); else every thread reads its own sequence's row.
+// Grid: (token blocks, layers); a block owns kPackTok consecutive tokens of one layer.  Its [heads][tokens] tile of
+// scores goes through shared memory: the loads are 16-byte, row-contiguous and all in flight at once (eight per
+// thread at 32 heads), and the per-token walk over the heads afterwards reads shared memory without conflicts.
+// The thresholds of the block's sequence sit in shared memory when all its tokens belong to one sequence (always,
+// with one sequence per batch); else every thread reads its own sequence's row.
+constexpr int kPackTok = 128;
+
 template <bool kImportance>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(kPackTok)
 signature_pack_kernel(Shape s, const float* __restrict__ scores, const float* __restrict__ theta,
-                      uint32_t* __restrict__ sigs, double* __restrict__ importance) {
+                      uint32_t* __restrict__ sigs, double* __restrict__ importance, int vec_ok) {
+  extern __shared__ float4 tile4[];                   // [Hq][kPackTok] float
+  float* tile = reinterpret_cast<float*>(tile4);
   __shared__ float th_sh[128];
   const int layer = blockIdx.y;
-  const int tok0 = blockIdx.x * 256, tok = tok0 + threadIdx.x;
-  const int seq0 = seq_of_token(s.cu_seqlens, s.n_seqs, tok0);
-  const bool one_seq = min(tok0 + 256, s.T) <= __ldg(s.cu_seqlens + seq0 + 1);
-  if (one_seq) {
-    if (threadIdx.x < s.Hq) th_sh[threadIdx.x] = __ldg(theta + ((size_t)layer * s.n_seqs + seq0) * s.Hq + threadIdx.x);
-    __syncthreads();
+  const int tok0 = blockIdx.x * kPackTok, tok = tok0 + threadIdx.x;
+  const int n_tok = min(kPackTok, s.T - tok0);
+  const float* base = scores + (size_t)layer * s.Hq * s.T + tok0;
+  if (vec_ok && n_tok == kPackTok) {                  // rows start on 16-byte boundaries
+#pragma unroll 8
+    for (int i = threadIdx.x; i < s.Hq * (kPackTok / 4); i += kPackTok) {
+      const int h = i / (kPackTok / 4), c = i % (kPackTok / 4);
+      tile4[i] = __ldg(reinterpret_cast<const float4*>(base + (size_t)h * s.T) + c);
+    }
+  } else {
+#pragma unroll 8
+    for (int h = 0; h < s.Hq; ++h)
+      tile[h * kPackTok + threadIdx.x] = (int)threadIdx.x < n_tok ? __ldg(base + (size_t)h * s.T + threadIdx.x) : 0.f;
   }
-  if (tok >= s.T) return;
+  const int seq0 = seq_of_token(s.cu_seqlens, s.n_seqs, tok0);
+  const bool one_seq = tok0 + n_tok <= __ldg(s.cu_seqlens + seq0 + 1);
+  if (one_seq)
+    for (int h = threadIdx.x; h < s.Hq; h += kPackTok) th_sh[h] = __ldg(theta + ((size_t)layer * s.n_seqs + seq0) * s.Hq + h);
+  __syncthreads();
+  if ((int)threadIdx.x >= n_tok) return;
   const float* th = one_seq ? th_sh
                             : theta + ((size_t)layer * s.n_seqs + seq_of_token(s.cu_seqlens, s.n_seqs, tok)) * s.Hq;
-  const float* sc = scores + (size_t)layer * s.Hq * s.T + tok;
+  const float* col = tile + threadIdx.x;
   uint32_t* out = sigs + ((size_t)layer * s.T + tok) * s.W;
   double total = 0.0, group = 0.0;
   int in_group = 0;
   for (int w = 0; w < s.W; ++w) {
     uint32_t word = 0;
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {             // 16 loads in flight at a time
-      const int h0 = 32 * w + 16 * half;
-      float v[16];
-#pragma unroll
-      for (int b = 0; b < 16; ++b) v[b] = h0 + b < s.Hq ? __ldg(sc + (size_t)(h0 + b) * s.T) : 0.f;
-#pragma unroll
-      for (int b = 0; b < 16; ++b)
-        if (h0 + b < s.Hq) word |= (uint32_t)(v[b] >= th[h0 + b]) << (16 * half + b);
+    const int nb = min(32, s.Hq - 32 * w);
+#pragma unroll 8
+    for (int b = 0; b < nb; ++b) {
+      const float v = col[(32 * w + b) * kPackTok];
+      word |= (uint32_t)(v >= th[32 * w + b]) << b;
       if constexpr (kImportance) {
-#pragma unroll
-        for (int b = 0; b < 16; ++b) {
-          if (h0 + b < s.Hq) {
-            group = __dadd_rn(group, (double)v[b]);
-            if (++in_group == s.G) { total = __dadd_rn(total, group); group = 0.0; in_group = 0; }
-          }
-        }
+        group = __dadd_rn(group, (double)v);
+        if (++in_group == s.G) { total = __dadd_rn(total, group); group = 0.0; in_group = 0; }
       }
     }
     out[w] = word;
@@ -270,7 +290,7 @@ int launch_signature(const Shape& s, const float* scores, const int32_t* sig_kee
     const int m = s.max_seqlen;
     if (m <= 2048) launch_theta<256, 8>(s, scores, sig_keep, theta, blocks, stream);
     else if (m <= 4096) launch_theta<256, 16>(s, scores, sig_keep, theta, blocks, stream);
-    else if (m <= 8192) launch_theta<256, 32>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 8192) launch_theta<KVC_THETA_T8K, 8192 / KVC_THETA_T8K>(s, scores, sig_keep, theta, blocks, stream);
     else if (m <= 16384) launch_theta<512, 32>(s, scores, sig_keep, theta, blocks, stream);
     else if (m <= 32768) launch_theta<1024, 32>(s, scores, sig_keep, theta, blocks, stream);
     else {
@@ -285,11 +305,19 @@ int launch_signature(const Shape& s, const float* scores, const int32_t* sig_kee
     if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
     th = theta;
   }
-  const dim3 grid((unsigned)((s.T + 255) / 256), (unsigned)s.n_layers);
-  if (importance)
-    signature_pack_kernel<true><<<grid, 256, 0, stream>>>(s, scores, th, sigs, importance);
-  else
-    signature_pack_kernel<false><<<grid, 256, 0, stream>>>(s, scores, th, sigs, nullptr);
+  const dim3 grid((unsigned)((s.T + kPackTok - 1) / kPackTok), (unsigned)s.n_layers);
+  const size_t dyn = (size_t)s.Hq * kPackTok * sizeof(float);
+  // 16-byte loads need every (layer, head) row to start on a 16-byte boundary
+  const int vec_ok = s.T % 4 == 0 && reinterpret_cast<uintptr_t>(scores) % 16 == 0;
+  if (importance) {
+    if (dyn > 48 * 1024 && cudaFuncSetAttribute(signature_pack_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+      return KVCRUSH_ERR_CUDA;
+    signature_pack_kernel<true><<<grid, kPackTok, dyn, stream>>>(s, scores, th, sigs, importance, vec_ok);
+  } else {
+    if (dyn > 48 * 1024 && cudaFuncSetAttribute(signature_pack_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+      return KVCRUSH_ERR_CUDA;
+    signature_pack_kernel<false><<<grid, kPackTok, dyn, stream>>>(s, scores, th, sigs, nullptr, vec_ok);
+  }
   return check_launch();
 }
 
