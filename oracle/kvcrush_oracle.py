@@ -60,6 +60,13 @@ because it gives no formula for them:
 Decode step (``decode_update``): the cumulative attention of H2O goes on while tokens are generated; one new query
 adds its softmax row over the cached keys.  PARITY UNPINNED by this paper (it describes the baseline in a sentence).
 
+Clustering baseline (``kmeans_select``; ablation "KMeans vs KVCrush", Fig. 3: k-means with 100 iterations in the place
+of the anchor / bucket grouping): Lloyd's algorithm on the binary head vectors of the tokens that are not important,
+k = B_representative, in exact rational arithmetic.  PARITY UNPINNED by the paper, which names the method and the
+iteration count only: the initial centroids (the vectors at evenly spaced ranks of the grouped tokens), ties to the
+lower cluster, empty clusters keeping their centroid, and the unused part of the budget going to the next most
+important tokens are this file's readings.
+
 Chunk- and page-granular eviction (Sec. 4.3.4: chunks of 8 tokens; Sec. 4.3.5: pages of 32 tokens): the
 paper gives two sentences - the baseline sums the attention weights over a page, and the
 binary vector of a page is the concatenation of the head vectors of its tokens.  Everything
@@ -356,6 +363,88 @@ def select(scores32: np.ndarray, sig: np.ndarray, b_imp: int, b_rep: int, n_kv_h
         reps = np.asarray([representative(srt[bounds[i]:bounds[i + 1]], sig[srt[bounds[i]:bounds[i + 1]]], Hq)
                            for i in range(b_rep)], dtype=np.int64)
     kept = np.sort(np.concatenate([imp, reps]))
+    kind = np.zeros(kept.shape[0], dtype=np.uint8)
+    kind[np.isin(kept, reps)] = 1
+    return kept, kind
+
+
+# ---------------------------------------------------------------------------
+# Clustering baseline: k-means in the place of Algorithm 2's grouping (ablation "KMeans vs KVCrush", Fig. 3)
+# ---------------------------------------------------------------------------
+
+def kmeans_assign(bits: np.ndarray, cnt: np.ndarray, m: np.ndarray) -> np.ndarray:
+    """Nearest centroid of every 0/1 row of ``bits`` [N, H]; centroid c is cnt[c] / m[c] (per-bit mean of m[c]
+    vectors).  Squared Euclidean distance  sum_h (b_h - n_h/m)^2 = (sum_h n_h^2 + m * sum_{h: b_h=1} (m - 2 n_h)) / m^2
+    is compared as an exact fraction (integers, cross-multiplied); ties go to the lower cluster index."""
+    N, k = bits.shape[0], cnt.shape[0]
+    out = np.zeros(N, dtype=np.int64)
+    S = [int((cnt[c].astype(object) ** 2).sum()) for c in range(k)]
+    wgt = [[int(m[c]) - 2 * int(x) for x in cnt[c]] for c in range(k)]
+    for t in range(N):
+        hs = np.nonzero(bits[t])[0]
+        best_num, best_den, best_c = None, None, -1
+        for c in range(k):
+            mc = int(m[c])
+            num = S[c] + mc * sum(wgt[c][h] for h in hs)        # distance = num / mc^2
+            den = mc * mc
+            if best_c < 0 or num * best_den < best_num * den:
+                best_num, best_den, best_c = num, den, c
+        out[t] = best_c
+    return out
+
+
+def kmeans_select(scores32: np.ndarray, sig: np.ndarray, b_imp: int, b_rep: int, n_kv_heads: int,
+                  iterations: int = 100, keep_recent: int = 0, keep_initial: int = 0):
+    """Kept token ids (ascending) and their kind when k-means takes the place of Algorithm 2's grouping.
+
+    The important set is that of ``select``.  The other tokens (ascending, N of them) are clustered into
+    k = b_rep clusters by Lloyd's algorithm on their binary head vectors: the initial centroids are the vectors at
+    ranks floor(i*N/k); an iteration assigns every vector to its nearest centroid (``kmeans_assign``) and replaces
+    each centroid by the per-bit mean of its members (a cluster without members keeps its centroid).  After
+    ``iterations`` iterations one more assignment fixes the members; every cluster that has members contributes
+    the member closest to its centroid (``representative``'s integer cost against that centroid, ties to the
+    lower token).  Budget that empty clusters leave unused goes to the grouped tokens of largest importance that
+    are not representatives (kind 0, like the important set)."""
+    Hq, L = scores32.shape
+    if b_imp + b_rep >= L:
+        return np.arange(L, dtype=np.int64), np.zeros(L, dtype=np.uint8)
+    I = importance(scores32, n_kv_heads)
+    if keep_recent > 0 or keep_initial > 0:
+        I = I.copy()
+        I[max(0, L - keep_recent):] = np.inf
+        I[:min(L, keep_initial)] = np.inf
+    imp = top_important(I, b_imp)
+    is_imp = np.zeros(L, dtype=bool)
+    is_imp[imp] = True
+    reps = np.zeros(0, dtype=np.int64)
+    fill = np.zeros(0, dtype=np.int64)
+    if b_rep > 0:
+        cand = np.nonzero(~is_imp)[0]
+        N, k = cand.shape[0], b_rep
+        bits = unpack_bits(sig[cand], Hq).astype(np.int64)
+        cnt = bits[[(i * N) // k for i in range(k)]].copy()
+        m = np.ones(k, dtype=np.int64)
+        for _ in range(iterations):
+            assign = kmeans_assign(bits, cnt, m)
+            for c in range(k):
+                members = assign == c
+                if members.any():
+                    cnt[c] = bits[members].sum(axis=0)
+                    m[c] = int(members.sum())
+        assign = kmeans_assign(bits, cnt, m)
+        rep_list = []
+        for c in range(k):
+            members = np.nonzero(assign == c)[0]
+            if members.shape[0] == 0:
+                continue
+            cost = (bits[members] * (m[c] - 2 * cnt[c])[None, :]).sum(axis=1)
+            rep_list.append(int(cand[members[np.lexsort((cand[members], cost))[0]]]))
+        reps = np.asarray(sorted(rep_list), dtype=np.int64)
+        shortfall = k - reps.shape[0]
+        if shortfall > 0:
+            rest = np.setdiff1d(cand, reps)
+            fill = rest[top_important(I[rest], shortfall)]
+    kept = np.sort(np.concatenate([imp, reps, fill]))
     kind = np.zeros(kept.shape[0], dtype=np.uint8)
     kind[np.isin(kept, reps)] = 1
     return kept, kind

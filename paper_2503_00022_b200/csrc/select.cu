@@ -37,13 +37,6 @@ __device__ __forceinline__ unsigned long long importance_key(double v, int t, in
   return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
 }
 
-// floor(b * N / R) for N = q_nr * R + r_nr, 0 <= b <= R < 2^18: b * q_nr + floor(b * r_nr / R), in 32 bits when it fits.
-__device__ __forceinline__ int bucket_lo(int b, int q_nr, int r_nr, int R) {
-  const unsigned long long p = (unsigned long long)(unsigned)b * (unsigned)r_nr;
-  const unsigned frac = R < 65536 ? (unsigned)p / (unsigned)R : (unsigned)(p / (unsigned)R);
-  return b * q_nr + (int)frac;
-}
-
 __global__ void __launch_bounds__(256)
 importance_kernel(Shape s, const float* __restrict__ scores, int keep_initial, int keep_recent,
                   unsigned long long* __restrict__ keys) {
@@ -278,11 +271,20 @@ select_segment_kernel(Shape s, SelectArgs a) {
       while (gw < m_max) gw <<= 1;
       const int per_warp = 32 / gw, sub = lane / gw, j = lane - sub * gw;
       const unsigned gmask = (0xFFFFFFFFu >> (32 - gw)) << (sub * gw);
-      for (int b0 = warp * per_warp; b0 < b_rep; b0 += kWarps * per_warp) {
-        const int bkt = b0 + sub;
+      // bucket b starts at b*q_nr + frac with b*r_nr = frac*R + rem.  Divisions are slow, so each lane divides once
+      // for its first bucket and then steps exactly by the warp's stride of kWarps*per_warp buckets.
+      const int first_bkt = warp * per_warp + sub, stride_b = kWarps * per_warp;
+      const unsigned long long p0 = (unsigned long long)(unsigned)first_bkt * (unsigned)r_nr;
+      const unsigned long long ps = (unsigned long long)(unsigned)stride_b * (unsigned)r_nr;
+      int frac = (int)(p0 / (unsigned)b_rep), rem = (int)(p0 - (unsigned long long)frac * (unsigned)b_rep);
+      const int step_q = (int)(ps / (unsigned)b_rep), step_r = (int)(ps - (unsigned long long)step_q * (unsigned)b_rep);
+      for (int bkt = first_bkt; bkt - sub < b_rep; bkt += stride_b) {
         const bool live = bkt < b_rep;
-        const int lo = live ? bucket_lo(bkt, q_nr, r_nr, b_rep) : 0;
-        const int m = live ? bucket_lo(bkt + 1, q_nr, r_nr, b_rep) - lo : 0;
+        const int lo = live ? bkt * q_nr + frac : 0;
+        const int m = live ? q_nr + (rem + r_nr >= b_rep ? 1 : 0) : 0;       // the next bucket's frac is one larger
+        frac += step_q;
+        rem += step_r;
+        if (rem >= b_rep) { rem -= b_rep; ++frac; }
         const bool member = j < m;
         const int t = member ? sorted[lo + j] : 0;
         uint32_t mine[4] = {0u, 0u, 0u, 0u};
