@@ -470,6 +470,34 @@ def run_ours(args, w):
     graph_ms = max_over_ranks(e0.elapsed_time(e1), dev, world) / args.steps
     cp.check_status()
 
+    # ---- the clustering baseline of the paper's ablation (k-means, 100 iterations, in the place of Algorithm 2's grouping)
+    # timed beside the selection stage on the same scores and signatures ----
+    kmeans = None
+    if args.kmeans and not args.page_size:
+        K = int(b_rep.max())
+        km_ws = torch.empty(max(256, B.kvcrush_kmeans_workspace_size(prob, K)), dtype=torch.uint8, device=dev)
+        km_idx, km_kind = torch.empty_like(cp.idx), torch.empty_like(cp.kind)
+        sc_sel = cp.pooled if cp.pooled is not None else cp.scores
+        def km():
+            B.kvcrush_kmeans_select(prob, sc_sel, cp.sigs, cp.budget_imp, cp.budget_rep, K, args.kmeans, cp.cu_kept,
+                                    km_idx, kind=km_kind, keep_initial=keep_initial, keep_recent=keep_recent,
+                                    workspace=km_ws, status=cp.status)
+        km()
+        torch.cuda.synchronize()
+        cp.check_status()
+        reps = max(1, min(args.steps, 3))
+        e0.record()
+        for _ in range(reps):
+            km()
+        e1.record()
+        torch.cuda.synchronize()
+        km_ms = e0.elapsed_time(e1) / reps
+        kmeans = {"iterations": args.kmeans, "ms": km_ms, "select_ms": float(stage_ms[2]), "ratio_to_select": km_ms / float(stage_ms[2]),
+                  "ratio_to_whole_pass": km_ms / ms_per_step,
+                  "agreement_with_kvcrush": float((torch.isin(km_idx, cp.idx).float().mean()).item()) if w.n_layers * w.n_seqs == 1 else None,
+                  "note": "k-means over the same binary head vectors, k = B_representative clusters per (layer, sequence)"}
+        del km_ws
+
     # ---- end to end through host buffers: H2D of the step's inputs, D2H of the kept set and reduced cache ----
     # Layers are independent, so the pass runs in chunks of layers: chunk c+1 is copied in (one stream) while
     # chunk c is compressed (the timed stream) and chunk c-1's kept indices and reduced cache are copied out
@@ -620,7 +648,7 @@ def run_ours(args, w):
                 "overlap": "H2D, compute and D2H of consecutive layer chunks on three streams"},
         "lse_supplied": {"ms_per_step": lse_ms, "value": whole_job_value(w.total_tokens, world, lse_ms), "unit": UNIT,
                          "note": "row log-sum-exp given by the caller: one score sweep instead of two"},
-        "sustained": sus,
+        "sustained": sus, "kmeans_baseline": kmeans,
         "gpu_launches": launches_per_step * args.steps,
         "gpu_launches_per_step": launches_per_step,
         "clocks": clocks,
@@ -639,6 +667,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--layers", type=int, default=0, help="run only this many layers of the workload (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kmeans", type=int, default=0,
+                    help="also time the k-means clustering baseline with this many iterations (the paper's ablation uses 100)")
     ap.add_argument("--sustained-s", type=float, default=4.0,
                     help="also loop the pass for at least this many seconds (0 = skip); the roofline fraction is taken there")
     ap.add_argument("--window", type=int, default=0,

@@ -58,6 +58,7 @@ extern "C" {
 /* status_dev[0] values */
 #define KVCRUSH_DEV_OK             0
 #define KVCRUSH_DEV_TIMEOUT        1     /* a bounded wait on a barrier ran out */
+#define KVCRUSH_DEV_BUDGET         2     /* kvcrush_kmeans_select: a budget_rep above max_budget_rep (status[2] = segment) */
 
 /* element types */
 #define KVCRUSH_BF16  0
@@ -308,6 +309,34 @@ int kvcrush_compact_pages(const kvcrush_problem_t* problem, const kvcrush_tensor
 int kvcrush_compact_scores(const kvcrush_problem_t* problem, const float* scores_in_dev, int page_size,
                            const int32_t* cu_kept_dev, const int32_t* idx_dev, int64_t total_kept,
                            float* scores_out_dev, int64_t out_tokens, int32_t* status_dev, void* stream);
+
+/*
+ * Clustering baseline of the ablation "KMeans vs KVCrush" (Experiments, Ablation Study, Fig. 3: k-means with 100
+ * iterations in the place of Algorithm 2's grouping, about 200 % more inference latency than H2O against less than
+ * 0.5 % for KVCrush).  Not a stage of the pass: it is here so that a conventional clustering of the same binary head
+ * vectors can be timed beside kvcrush_select.  Same arguments, outputs and important set as kvcrush_select; the
+ * other tokens (ascending, N of them) are grouped by Lloyd's algorithm instead of by Hamming distance to an anchor:
+ *   k = budget_rep clusters; initial centroids = the vectors at ranks floor(i*N/k) of the grouped tokens;
+ *   an iteration assigns every vector to the centroid at the smallest squared Euclidean distance (compared exactly,
+ *   as integer fractions; ties: lower cluster) and replaces every centroid by the per-bit mean of its members (a
+ *   cluster without members keeps its centroid); after `iterations` iterations one more assignment fixes the members;
+ *   every cluster with members gives the member closest to its centroid (ties: lower token), kind 1;
+ *   budget that empty clusters leave unused goes to the most important of the remaining tokens, kind 0.
+ * The paper gives the method's name and iteration count only; initialisation, tie rules and the treatment of empty
+ * clusters are this library's.
+ *   max_budget_rep   host value: no budget_rep of the call exceeds it (sizes the workspace); a larger budget is
+ *                    reported as KVCRUSH_DEV_BUDGET through status_dev and that segment is left unwritten
+ *   iterations       >= 0 (the paper's figure uses 100)
+ *   workspace        kvcrush_kmeans_workspace_size(problem, max_budget_rep) bytes
+ * Sequences longer than 32768 tokens, or with n_q_heads * max_seqlen^4 >= 2^66 (the exact comparison works in 64-bit
+ * integers), return KVCRUSH_ERR_UNSUPPORTED.
+ */
+int kvcrush_kmeans_workspace_size(const kvcrush_problem_t* problem, int max_budget_rep, size_t* bytes);
+int kvcrush_kmeans_select(const kvcrush_problem_t* problem, const float* scores_dev, const double* importance_dev,
+                          const uint32_t* sigs_dev, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+                          int max_budget_rep, int iterations, int keep_initial, int keep_recent,
+                          const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev, int32_t* n_kept_dev,
+                          void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
 /*
  * Stage 2 without caller-provided scratch (the paper has no counterpart; this is a packaging

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_PKG, "libkvcrush.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_WORKSPACE, ERR_CUDA = 0, -1, -2, -3, -4, -5
 ERR_STATIC_LIMIT = -6
 STATIC_THETA_MAX = 65536
-DEV_OK, DEV_TIMEOUT = 0, 1
+DEV_OK, DEV_TIMEOUT, DEV_BUDGET = 0, 1, 2
 BF16, FP16, FP32 = 0, 1, 2
 STAGE_SCORE, STAGE_SIGNATURE, STAGE_SELECT, STAGE_COMPACT = 0, 1, 2, 3
 ANCHOR_ALTERNATE, ANCHOR_MEAN, ANCHOR_EXPLICIT = 0, 1, 2
@@ -29,7 +29,7 @@ SCORE_AUTO, SCORE_SIMT, SCORE_TENSOR = 0, 1, 2
 EXPORTS = ("kvcrush_workspace_size", "kvcrush_score", "kvcrush_signature", "kvcrush_select",
            "kvcrush_compact", "kvcrush_strerror", "kvcrush_version", "kvcrush_signature_static",
            "kvcrush_pool_scores", "kvcrush_select_pages", "kvcrush_compact_pages", "kvcrush_score_decode",
-           "kvcrush_compact_scores")
+           "kvcrush_compact_scores", "kvcrush_kmeans_workspace_size", "kvcrush_kmeans_select")
 
 
 class ProblemStruct(ctypes.Structure):
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.kvcrush_signature.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_select.argtypes = [P, vp, vp, vp, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_pool_scores.argtypes = [P, vp, i32, vp, vp, vp]
+        L.kvcrush_kmeans_workspace_size.argtypes = [P, i32, ctypes.POINTER(sz)]
+        L.kvcrush_kmeans_select.argtypes = [P, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_compact.argtypes = [P, T, T, vp, vp, i64, T, T, vp, vp]
         L.kvcrush_select_pages.argtypes = [P, vp, vp, vp, i32, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         L.kvcrush_compact_pages.argtypes = [P, T, T, i32, vp, vp, i64, T, T, vp, vp]
@@ -204,6 +206,25 @@ def kvcrush_select(problem: Problem, scores, sigs, budget_imp, budget_rep, cu_ke
                                 int(keep_recent), _ptr(cu_kept),
                                 _ptr(idx), _ptr(kind), _ptr(n_kept), _ptr(workspace), ws_bytes, _ptr(status),
                                 _stream() if stream is None else stream), "kvcrush_select")
+
+
+def kvcrush_kmeans_workspace_size(problem: Problem, max_budget_rep: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().kvcrush_kmeans_workspace_size(problem.ref, int(max_budget_rep), ctypes.byref(out)),
+           "kvcrush_kmeans_workspace_size")
+    return int(out.value)
+
+
+def kvcrush_kmeans_select(problem: Problem, scores, sigs, budget_imp, budget_rep, max_budget_rep: int, iterations: int,
+                          cu_kept, idx, *, importance=None, kind=None, n_kept=None, keep_initial=0, keep_recent=0,
+                          workspace=None, status=None, stream: Optional[int] = None) -> None:
+    """The clustering baseline: k-means on the binary head vectors in the place of kvcrush_select's grouping."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().kvcrush_kmeans_select(problem.ref, _ptr(scores), _ptr(importance), _ptr(sigs), _ptr(budget_imp),
+                                       _ptr(budget_rep), int(max_budget_rep), int(iterations), int(keep_initial),
+                                       int(keep_recent), _ptr(cu_kept), _ptr(idx), _ptr(kind), _ptr(n_kept),
+                                       _ptr(workspace), ws_bytes, _ptr(status),
+                                       _stream() if stream is None else stream), "kvcrush_kmeans_select")
 
 
 def kvcrush_pool_scores(problem: Problem, scores_in, kernel: int, scores_out, *, status=None,

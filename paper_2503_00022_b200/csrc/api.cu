@@ -205,6 +205,36 @@ int kvcrush_select(const kvcrush_problem_t* problem, const float* scores_dev, co
                        workspace, static_cast<cudaStream_t>(stream));
 }
 
+int kvcrush_kmeans_workspace_size(const kvcrush_problem_t* problem, int max_budget_rep, size_t* bytes) {
+  Shape s;
+  if (!bytes || max_budget_rep < 0) return KVCRUSH_ERR_INVALID_ARG;
+  const int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  *bytes = kmeans_workspace_bytes(s, max_budget_rep);
+  return KVCRUSH_OK;
+}
+
+int kvcrush_kmeans_select(const kvcrush_problem_t* problem, const float* scores_dev, const double* importance_dev,
+                          const uint32_t* sigs_dev, const int32_t* budget_imp_dev, const int32_t* budget_rep_dev,
+                          int max_budget_rep, int iterations, int keep_initial, int keep_recent,
+                          const int32_t* cu_kept_dev, int32_t* idx_dev, uint8_t* kind_dev, int32_t* n_kept_dev,
+                          void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  Shape s;
+  const int rc = make_shape(problem, &s);
+  if (rc != KVCRUSH_OK) return rc;
+  if ((!scores_dev && !importance_dev) || !sigs_dev || !budget_imp_dev || !budget_rep_dev || !cu_kept_dev || !idx_dev ||
+      !status_dev)
+    return KVCRUSH_ERR_INVALID_ARG;
+  if (importance_dev && reinterpret_cast<uintptr_t>(importance_dev) % 8) return KVCRUSH_ERR_MISALIGNED;
+  if (max_budget_rep < 0 || iterations < 0 || keep_recent < 0 || keep_initial < 0) return KVCRUSH_ERR_INVALID_ARG;
+  if (!kmeans_supported(s)) return KVCRUSH_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < kmeans_workspace_bytes(s, max_budget_rep)) return KVCRUSH_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return KVCRUSH_ERR_MISALIGNED;
+  return launch_kmeans_select(s, scores_dev, importance_dev, sigs_dev, budget_imp_dev, budget_rep_dev, max_budget_rep,
+                              iterations, keep_initial, keep_recent, cu_kept_dev, idx_dev, kind_dev, n_kept_dev,
+                              workspace, status_dev, static_cast<cudaStream_t>(stream));
+}
+
 int kvcrush_compact(const kvcrush_problem_t* problem, const kvcrush_tensor_t* K, const kvcrush_tensor_t* V,
                     const int32_t* cu_kept_dev, const int32_t* idx_dev, int64_t total_kept,
                     const kvcrush_tensor_t* K_out, const kvcrush_tensor_t* V_out,

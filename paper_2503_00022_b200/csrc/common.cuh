@@ -26,7 +26,7 @@ struct TensorView {
 inline int elt_bytes(int dtype) { return dtype == KVCRUSH_FP32 ? 4 : 2; }
 
 // kernel ids written to status[1]
-enum KernelId { KID_SCORE_LSE = 1, KID_SCORE_COLSUM = 2 };
+enum KernelId { KID_SCORE_LSE = 1, KID_SCORE_COLSUM = 2, KID_KMEANS = 3 };
 
 __device__ __forceinline__ void report(int32_t* status, int code, int kid, int a, int b) {
   if (atomicCAS(status, 0, code) == 0) {
@@ -89,6 +89,18 @@ int launch_select(const Shape& s, const float* scores, const double* importance,
 // Order-preserving 64-bit keys of the token importance I(t), [n_layers][T] (first kernel of the selection stages).
 int launch_importance(const Shape& s, const float* scores, int keep_initial, int keep_recent,
                       unsigned long long* keys, cudaStream_t stream);
+
+// The same keys from an importance array [n_layers][T] the caller supplies.
+int launch_importance_keys(const Shape& s, const double* importance, int keep_initial, int keep_recent,
+                           unsigned long long* keys, cudaStream_t stream);
+
+// Clustering baseline (k-means in the place of Algorithm 2's grouping); max_budget_rep bounds every budget_rep.
+size_t kmeans_workspace_bytes(const Shape& s, int max_budget_rep);
+bool kmeans_supported(const Shape& s);
+int launch_kmeans_select(const Shape& s, const float* scores, const double* importance, const uint32_t* sigs,
+                         const int32_t* budget_imp, const int32_t* budget_rep, int max_budget_rep, int iterations,
+                         int keep_initial, int keep_recent, const int32_t* cu_kept, int32_t* idx, uint8_t* kind,
+                         int32_t* n_kept, void* ws, int32_t* status, cudaStream_t stream);
 
 // Page-granular selection and gather (a page = page_size consecutive tokens of one sequence).
 constexpr int kMaxPagesPerSeq = 8192;      // pages of one sequence the page kernel holds in shared memory

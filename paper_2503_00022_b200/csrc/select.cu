@@ -390,6 +390,13 @@ int launch_importance(const Shape& s, const float* scores, int keep_initial, int
   return check_launch();
 }
 
+int launch_importance_keys(const Shape& s, const double* importance, int keep_initial, int keep_recent,
+                           unsigned long long* keys, cudaStream_t stream) {
+  const size_t n = (size_t)s.n_layers * s.T;
+  importance_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, importance, keep_initial, keep_recent, keys);
+  return check_launch();
+}
+
 size_t select_workspace_bytes(const Shape& s) {
   const size_t n = (size_t)s.n_layers * s.T;
   return ((n * 8 + 255) / 256) * 256 + ((n * 4 + 255) / 256) * 256;
