@@ -141,6 +141,16 @@ class ClockSampler:
             return None
         return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
 
+    def series(self):
+        """(wall time, SM MHz, board W) of every sample taken so far."""
+        out = []
+        for t, r in self.rows:
+            try:
+                out.append((t, float(r[0]), float(r[2])))
+            except (ValueError, IndexError):
+                continue
+        return out
+
 
 # ---------------------------------------------------------------------------------------------
 # input staging
@@ -414,9 +424,26 @@ def run_ours(args, w):
         cp.check_status()
         sus_ms = max_over_ranks(e0.elapsed_time(e1), dev, world) / n_sus
         half = n_sus // 2                                                     # settled part of the loop
-        sus_score_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in ev_s[half:]]))
+        score_each = [a_.elapsed_time(b_) for a_, b_ in ev_s]
+        sus_score_ms = float(np.mean(score_each[half:]))
         sus = dict(steps=n_sus, seconds=sus_ms * n_sus * 1e-3, ms_per_step=sus_ms, score_ms_settled=sus_score_ms,
                    clocks=clocks_s)
+        # the unchanged kernels against the clock they ran at: eight windows of the loop, each with the mean score-stage
+        # time of its steps, the median sampled SM clock and board power, and their product (Mcycles per step)
+        if sampler_s:
+            start = [e0.elapsed_time(a_) * 1e-3 for a_, _ in ev_s]            # device-time offset of every step
+            ser = sampler_s.series()
+            wins = []
+            span = sus["seconds"]
+            for i in range(8):
+                lo, hi = span * i / 8, span * (i + 1) / 8
+                ms_w = [m for m, t0_ in zip(score_each, start) if lo <= t0_ < hi]
+                mhz_w = [mhz for t_, mhz, _ in ser if lo <= t_ - t_b < hi]
+                pw_w = [pw for t_, _, pw in ser if lo <= t_ - t_b < hi]
+                if ms_w and mhz_w:
+                    wins.append({"t_s": round(lo, 2), "score_ms": float(np.mean(ms_w)), "sm_mhz": float(np.median(mhz_w)),
+                                 "board_w": float(np.median(pw_w)), "score_ms_x_ghz": float(np.mean(ms_w) * np.median(mhz_w) * 1e-3)})
+            sus["windows"] = wins
 
     # ---- the same pass when the caller already has the row log-sum-exp (a prefill attention kernel returns it):
     # the first sweep is skipped.  Reported beside the headline, never instead of it.

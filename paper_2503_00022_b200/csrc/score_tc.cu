@@ -68,6 +68,8 @@ struct PersistArgs {
   int max_blocks;          // ceil(max_seqlen / kBlockRows)
   int n_items;             // (sequence, stationary block) pairs of one (layer, head)
   int total_items;         // n_items * n_layers * Hq
+  int n_lh;                // n_layers * Hq
+  int tail_lh;             // the last tail_lh (layer, head) pairs are handed out heaviest item first across all of them
   int* counter;            // work counter, zero at launch
   int32_t* status;
   int withhold_first_item; // diagnostic: the producer warp fetches its first item and then stops before announcing
@@ -217,7 +219,17 @@ score_persist_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         break;
       }
       if (a.withhold_first_item) break;        // nothing is in flight: the consumers' bounded waits end the CTA
-      const int lh = idx / a.n_items, rank = idx - lh * a.n_items;
+      // (layer, head)-major order keeps the CTAs that run together on a few heads (their Q and K stay in L2); the
+      // last pairs are taken weight-major instead, so that the launch does not end with a few CTAs on the heaviest
+      // items of the last head while the others idle (a launch with few items is all tail)
+      int lh, rank;
+      const int head_part = (a.n_lh - a.tail_lh) * a.n_items;
+      if (idx < head_part) {
+        lh = idx / a.n_items; rank = idx - lh * a.n_items;
+      } else {
+        const int j = idx - head_part;
+        rank = j / a.tail_lh; lh = a.n_lh - a.tail_lh + (j - rank * a.tail_lh);
+      }
       int seq, blk, nblk;
       decode_item(s.cu_seqlens, s.n_seqs, a.max_blocks, rank, !kColsum, lane, seq, blk, nblk, kBlockRows, s.window);
       if (lane == 0) {
@@ -530,10 +542,16 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
   if (items_col == 0) return KVCRUSH_OK;
   if (items_col * s.n_layers * s.Hq > 0x7FFFFFFFLL) return KVCRUSH_ERR_UNSUPPORTED;
   if (cudaMemsetAsync(counters, 0, 2 * sizeof(int), stream) != cudaSuccess) return KVCRUSH_ERR_CUDA;
+  a.n_lh = s.n_layers * s.Hq;
+  auto tail_pairs = [&](long long items) {       // pairs whose items make up about four rounds of the grid
+    const long long t = (4LL * n_sms + items - 1) / items;
+    return (int)(t < a.n_lh ? t : a.n_lh);
+  };
   int rc;
   if (!lse_in) {
     a.lse2_out = lse2_ws; a.lse_nat_out = lse_out; a.counter = counters;
     a.n_items = (int)items_row; a.total_items = (int)(items_row * s.n_layers * s.Hq);
+    a.tail_lh = tail_pairs(items_row);
     rc = s.D > 64 ? launch_persist<128, false>(mq, mk, a, sw, n_sms, stream) : launch_persist<64, false>(mq, mk, a, sw, n_sms, stream);
     if (rc != KVCRUSH_OK) return rc;
     a.lse = lse2_ws; a.lse_mul = 1.f;
@@ -542,6 +560,7 @@ int launch_score_tensor(const Shape& s, const int32_t* cu_host, const TensorView
   }
   a.counter = counters + 1;
   a.n_items = (int)items_col; a.total_items = (int)(items_col * s.n_layers * s.Hq);
+  a.tail_lh = tail_pairs(items_col);
   return s.D > 64 ? launch_persist<128, true>(mq, mk, a, sw, n_sms, stream) : launch_persist<64, true>(mq, mk, a, sw, n_sms, stream);
 }
 

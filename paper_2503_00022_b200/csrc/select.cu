@@ -433,12 +433,15 @@ int launch_select(const Shape& s, const float* scores, const double* importance,
   if (!importance) {
     if (launch_importance(s, scores, keep_initial, keep_recent, keys, stream) != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
     a.keys = keys;
-  } else if (a.stage_keys) {
-    a.imp = importance; a.keep_initial = keep_initial; a.keep_recent = keep_recent;
-  } else {
-    importance_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, importance, keep_initial, keep_recent, keys);
-    if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
-    a.keys = keys;
+  }
+  if (importance) {
+    if (a.stage_keys) {
+      a.imp = importance; a.keep_initial = keep_initial; a.keep_recent = keep_recent;
+    } else {
+      importance_keys_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, importance, keep_initial, keep_recent, keys);
+      if (check_launch() != KVCRUSH_OK) return KVCRUSH_ERR_CUDA;
+      a.keys = keys;
+    }
   }
   if (dyn > 16 * 1024) {     // static + dynamic shared memory above the 48 KB default needs the opt-in
     cudaError_t e = cudaSuccess;

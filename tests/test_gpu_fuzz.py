@@ -19,17 +19,17 @@ def B():
     return binding
 
 
-def test_random_selection_problems_are_bit_exact(B):
+def _random_selection_cases(B, seed, n_cases, lengths, max_seqs):
     import torch
     dev = torch.device("cuda:0")
-    g = np.random.Generator(np.random.Philox(2024))
-    for case in range(36):
+    g = np.random.Generator(np.random.Philox(seed))
+    for case in range(n_cases):
         Hkv = int(g.choice([1, 2, 3, 8, 16]))
         Hq = Hkv * int(g.choice([1, 2, 4, 8]))
         if Hq > 128:
             Hq = Hkv
-        n_seqs = int(g.integers(1, 5))
-        seqlens = [int(g.choice([1, 2, 31, 32, 33, 64, 100, 257, 1000, 2100])) for _ in range(n_seqs)]
+        n_seqs = int(g.integers(1, max_seqs + 1))
+        seqlens = [int(g.choice(lengths)) for _ in range(n_seqs)]
         n_layers = int(g.integers(1, 3))
         ties = int(g.choice([0, 0, 2, 5]))
         mode = int(g.integers(0, 3))
@@ -68,6 +68,16 @@ def test_random_selection_problems_are_bit_exact(B):
                 seg = l * n_seqs + s
                 lo, hi = int(cp.cu_kept_host[seg]), int(cp.cu_kept_host[seg + 1])
                 assert np.array_equal(cp.kind[lo:hi].cpu().numpy(), kind), ctx
+                assert int(cp.n_kept[l, s]) == hi - lo, ctx
+
+
+def test_random_selection_problems_are_bit_exact(B):
+    _random_selection_cases(B, 2024, 36, [1, 2, 31, 32, 33, 64, 100, 257, 1000, 2100], 4)
+
+
+def test_random_selection_problems_with_long_segments_are_bit_exact(B):
+    # few long segments beside very short ones: several keys per thread in every sweep, buckets of all sizes
+    _random_selection_cases(B, 777, 20, [1, 40, 1024, 1025, 1500, 2100, 3000, 5000, 9000], 3)
 
 
 def test_random_score_problems_match_oracle_and_cuda_core_path(B):
