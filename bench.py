@@ -35,9 +35,13 @@ METRIC = "prompt tokens compressed/s (score+select+compact)"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg3_llama2_32l_8k"
 # dram__bytes_read + dram__bytes_write of one sweep launch per layer, from the ncu capture of the 2-layer case:
-# (276.0 + 276.7) MB / 2 sweeps / 2 layers.  Valid for the kernel source named in NCU_TRAFFIC_SOURCE only.
-NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP = 138.2e6
-NCU_TRAFFIC_SOURCE = "ncu capture of score_persist_kernel at commit ec18db7 (2 layers of the workload, scaled by the layer count)"
+# the column-sum sweep read 286.1 MB and wrote 5.5 MB for two layers.  Scaling by the layer count over-states the
+# full workload a little: the last 37 (layer, head) pairs of a launch are handed out across heads, which costs L2
+# reuse, and they are 37 of 64 pairs in the capture but 37 of 1024 in the full workload.  Valid for the kernel
+# source named in NCU_TRAFFIC_SOURCE only.
+NCU_DRAM_BYTES_PER_LAYER_PER_SWEEP = 145.8e6
+NCU_TRAFFIC_SOURCE = ("ncu capture of score_persist_kernel<128, colsum> at commit 8454247 (2 layers of the workload, scaled by the "
+                      "layer count: an upper bound, see profiles/)")
 
 
 def measured_peaks():
@@ -253,7 +257,6 @@ def workload_config(w: inputs.Workload, world: int, args, b_imp, b_rep):
             "keep_initial": args.keep_initial, "keep_recent": max(args.window, args.keep_recent)}
 
 
-REFERENCE_BUDGET_S = 450.0     # the whole --impl reference run (warm-up + steps) is sized to end within this
 
 
 def run_reference(args, w):
@@ -276,10 +279,10 @@ def run_reference(args, w):
     n_req = args.warmup + args.steps
     heads = 0                                              # whole layers
     steps, warmup = args.steps, args.warmup
-    if cal_s * rounds * n_req > REFERENCE_BUDGET_S:
+    if cal_s * rounds * n_req > args.reference_budget_s:
         heads = cal_heads if cal_heads < w.n_q_heads else 0
         per = cal_s if heads else cal_s * rounds
-        fit = max(1, int(REFERENCE_BUDGET_S / per))
+        fit = max(1, int(args.reference_budget_s / per))
         if fit < n_req:                                    # still too long: fewer steps, said in the line
             warmup = min(warmup, max(0, fit - 1) // 4)
             steps = max(1, min(steps, fit - warmup))
@@ -694,6 +697,9 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--layers", type=int, default=0, help="run only this many layers of the workload (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--reference-budget-s", type=float, default=450.0,
+                    help="--impl reference: the run (warm-up + steps) is sized to end within this many seconds; a whole pass "
+                         "of the oracle over every layer (--steps LAYERS --warmup 0) needs more")
     ap.add_argument("--kmeans", type=int, default=0,
                     help="also time the k-means clustering baseline with this many iterations (the paper's ablation uses 100)")
     ap.add_argument("--sustained-s", type=float, default=4.0,
