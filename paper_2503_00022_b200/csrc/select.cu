@@ -142,6 +142,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
   const unsigned long long* keys = a.keys ? a.keys + (size_t)layer * s.T + t0 : nullptr;
   const uint32_t* sig = a.sigs + ((size_t)layer * s.T + t0) * W;
   int32_t* sorted = a.sorted + (size_t)layer * s.T + t0;
+  uint32_t* sort_code = nullptr;         // per token: distance | position among the warp's tokens of that distance << 8
   {
     uint32_t* arena = dyn_smem + 2 * a.mask_words;
     if (a.stage_sorted) { sorted = reinterpret_cast<int32_t*>(arena); arena += a.stage_words; }
@@ -152,6 +153,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
     }
     if (a.stage_keys) {
       unsigned long long* ks = reinterpret_cast<unsigned long long*>(arena);
+      sort_code = reinterpret_cast<uint32_t*>(arena);      // the keys are dead once the important set is marked
       if (a.keys) {
         for (int i = tid; i < L; i += kThreads) ks[i] = keys[i];
       } else {
@@ -213,7 +215,9 @@ select_segment_kernel(Shape s, SelectArgs a) {
     _Pragma("unroll") for (int w = 0; w < 4; ++w) { anc[w] = w < W ? anchor_sh[w] : 0u; hm[w] = w < W ? head_mask(s.Hq, w) : 0u; }
     const int n_bins = s.Hq + 1;
 
-    // counting sort by (d, t): per-warp histograms over contiguous token ranges
+    // counting sort by (d, t): per-warp histograms over contiguous token ranges.  When there is room, the first
+    // sweep also notes every token's distance and its position among the warp's tokens of that distance, so that
+    // the second sweep is a plain scatter.
     for (int base = r_lo; base < r_hi; base += 32) {
       const int i = base + lane;
       const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
@@ -221,10 +225,15 @@ select_segment_kernel(Shape s, SelectArgs a) {
       if (cand)
         _Pragma("unroll") for (int w = 0; w < W; ++w) d += __popc((sig[(size_t)i * W + w] ^ anc[w]) & hm[w]);
       const unsigned voters = __ballot_sync(kFull, cand);
+      unsigned peers = 0;
       if (cand) {
-        const unsigned peers = __match_any_sync(voters, d);
-        if ((peers & lt_mask) == 0) warp_hist[warp][d] += __popc(peers);
+        peers = __match_any_sync(voters, d);
+        if (sort_code) sort_code[i] = (uint32_t)d | ((uint32_t)(warp_hist[warp][d] + __popc(peers & lt_mask)) << 8);
+      } else if (sort_code && i < r_hi) {
+        sort_code[i] = 0xFFFFFFFFu;
       }
+      __syncwarp();
+      if (cand && (peers & lt_mask) == 0) warp_hist[warp][d] += __popc(peers);
       __syncwarp();
     }
     __syncthreads();
@@ -239,21 +248,31 @@ select_segment_kernel(Shape s, SelectArgs a) {
       for (int b = 1; b <= n_bins; ++b) bin_base[b] += bin_base[b - 1];
     }
     __syncthreads();
-    for (int base = r_lo; base < r_hi; base += 32) {
-      const int i = base + lane;
-      const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
-      int d = 0;
-      if (cand)
-        _Pragma("unroll") for (int w = 0; w < W; ++w) d += __popc((sig[(size_t)i * W + w] ^ anc[w]) & hm[w]);
-      const unsigned voters = __ballot_sync(kFull, cand);
-      unsigned peers = 0;
-      if (cand) {
-        peers = __match_any_sync(voters, d);
-        sorted[bin_base[d] + warp_hist[warp][d] + __popc(peers & lt_mask)] = i;
+    if (sort_code) {
+      for (int i = r_lo + lane; i < r_hi; i += 32) {
+        const uint32_t c = sort_code[i];
+        if (c != 0xFFFFFFFFu) {
+          const int d = (int)(c & 0xFFu);
+          sorted[bin_base[d] + warp_hist[warp][d] + (int)(c >> 8)] = i;
+        }
       }
-      __syncwarp();
-      if (cand && (peers & lt_mask) == 0) warp_hist[warp][d] += __popc(peers);
-      __syncwarp();
+    } else {
+      for (int base = r_lo; base < r_hi; base += 32) {
+        const int i = base + lane;
+        const bool cand = i < r_hi && !((imp_mask[base >> 5] >> lane) & 1u);
+        int d = 0;
+        if (cand)
+          _Pragma("unroll") for (int w = 0; w < W; ++w) d += __popc((sig[(size_t)i * W + w] ^ anc[w]) & hm[w]);
+        const unsigned voters = __ballot_sync(kFull, cand);
+        unsigned peers = 0;
+        if (cand) {
+          peers = __match_any_sync(voters, d);
+          sorted[bin_base[d] + warp_hist[warp][d] + __popc(peers & lt_mask)] = i;
+        }
+        __syncwarp();
+        if (cand && (peers & lt_mask) == 0) warp_hist[warp][d] += __popc(peers);
+        __syncwarp();
+      }
     }
     __syncthreads();
 

@@ -217,10 +217,14 @@ __device__ __forceinline__ void mark_top_keys(const unsigned long long* keys, in
 __device__ __forceinline__ void emit_kept(const uint32_t* imp_mask, const uint32_t* rep_mask, int n_words,
                                           int32_t* out_idx, uint8_t* out_kind, Scratch& sc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int wpt = (n_words + kThreads - 1) / kThreads;      // mask words per thread, contiguous
-  const int w_lo = min(n_words, tid * wpt), w_hi = min(n_words, w_lo + wpt);
+  // every thread takes a contiguous run of mask BYTES (8 items each): with fewer words than threads a word-wise
+  // split would leave most threads idle and the others with up to 32 serial stores
+  const int n_bytes = 4 * n_words;
+  const int bpt = (n_bytes + kThreads - 1) / kThreads;
+  const int b_lo = min(n_bytes, tid * bpt), b_hi = min(n_bytes, b_lo + bpt);
+  auto byte_of = [](const uint32_t* mask, int b) -> uint32_t { return (mask[b >> 2] >> (8 * (b & 3))) & 0xFFu; };
   int cnt = 0;
-  for (int w = w_lo; w < w_hi; ++w) cnt += __popc(imp_mask[w] | rep_mask[w]);
+  for (int b = b_lo; b < b_hi; ++b) cnt += __popc(byte_of(imp_mask, b) | byte_of(rep_mask, b));
   int incl = cnt;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
@@ -232,14 +236,14 @@ __device__ __forceinline__ void emit_kept(const uint32_t* imp_mask, const uint32
   __syncthreads();
   int pos = incl - cnt;
   for (int w = 0; w < warp; ++w) pos += sc.warp_tot[w];
-  for (int w = w_lo; w < w_hi; ++w) {
-    const uint32_t rep = rep_mask[w];
-    uint32_t bits = imp_mask[w] | rep;
+  for (int b = b_lo; b < b_hi; ++b) {
+    const uint32_t rep = byte_of(rep_mask, b);
+    uint32_t bits = byte_of(imp_mask, b) | rep;
     while (bits) {
-      const int b = __ffs(bits) - 1;
+      const int k = __ffs(bits) - 1;
       bits &= bits - 1;
-      out_idx[pos] = 32 * w + b;
-      if (out_kind) out_kind[pos] = (rep >> b) & 1u;
+      out_idx[pos] = 8 * b + k;
+      if (out_kind) out_kind[pos] = (rep >> k) & 1u;
       ++pos;
     }
   }
