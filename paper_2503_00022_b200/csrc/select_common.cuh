@@ -30,6 +30,12 @@ __device__ __forceinline__ uint32_t head_mask(int Hq, int w) {
   return n >= 32 ? 0xFFFFFFFFu : ((1u << n) - 1u);
 }
 
+// Sum of tot[0 .. warp) for every thread of warp `warp`: one load per lane and a warp reduction instead of a serial
+// walk (the last warp would otherwise do 31 dependent loads).  n_warps <= 32.
+__device__ __forceinline__ int warps_before(const int* tot, int warp, int lane) {
+  return __reduce_add_sync(kFull, lane < warp ? tot[lane] : 0);
+}
+
 // Contiguous item range of a warp: a multiple of 32 items, so that mask words do not straddle warps.
 __device__ __forceinline__ void warp_range(int n, int warp, int& r_lo, int& r_hi) {
   const int n_words = (n + 31) >> 5;
@@ -68,7 +74,7 @@ __device__ __forceinline__ void find_digit_desc(const uint32_t* hist, int n_bins
   if (lane == 31) warp_tot[warp] = (int)incl;
   __syncthreads();
   uint32_t excl = incl - local;
-  for (int w = 0; w < warp; ++w) excl += (uint32_t)warp_tot[w];
+  excl += (uint32_t)warps_before(warp_tot, warp, lane);
   if (tid < n_act && excl < k_rem && k_rem <= excl + local) {
     uint32_t acc = excl;
     for (int j = 0; j < per; ++j) {
@@ -198,7 +204,7 @@ __device__ __forceinline__ void mark_top_keys(const unsigned long long* keys, in
   if (lane == 0) sc.warp_tot[warp] = n_eq;
   __syncthreads();
   int eq_before = 0;
-  for (int w = 0; w < warp; ++w) eq_before += sc.warp_tot[w];
+  eq_before += warps_before(sc.warp_tot, warp, lane);
   for (int base_i = r_lo; base_i < r_hi; base_i += 32) {
     const int i = base_i + lane;
     const unsigned long long key = i < r_hi ? keys[i] : 0ull;
@@ -235,7 +241,7 @@ __device__ __forceinline__ void emit_kept(const uint32_t* imp_mask, const uint32
   if (lane == 31) sc.warp_tot[warp] = incl;
   __syncthreads();
   int pos = incl - cnt;
-  for (int w = 0; w < warp; ++w) pos += sc.warp_tot[w];
+  pos += warps_before(sc.warp_tot, warp, lane);
   for (int b = b_lo; b < b_hi; ++b) {
     const uint32_t rep = byte_of(rep_mask, b);
     uint32_t bits = byte_of(imp_mask, b) | rep;
