@@ -91,9 +91,9 @@ __device__ __forceinline__ void find_digit_desc(const uint32_t* hist, int n_bins
 }
 
 // One warp ranks at most 32 candidates held one per lane (lanes >= n hold nothing): returns in every lane the
-// k_rem-th largest value and sets k_out to the rank left among the candidates equal to it.
+// k_rem-th largest value, sets k_out to the rank left among the candidates equal to it and n_equal to their number.
 __device__ __forceinline__ unsigned long long warp_rank_select(unsigned long long v, int n, uint32_t k_rem, int lane,
-                                                               uint32_t& k_out) {
+                                                               uint32_t& k_out, uint32_t& n_equal) {
   uint32_t gt = 0, ge = 0;
   for (int j = 0; j < n; ++j) {
     const unsigned long long o = __shfl_sync(kFull, v, j);
@@ -103,7 +103,9 @@ __device__ __forceinline__ unsigned long long warp_rank_select(unsigned long lon
   const bool hit = lane < n && gt < k_rem && k_rem <= ge;
   const unsigned who = __ballot_sync(kFull, hit);
   const int src = __ffs(who) - 1;                     // equal candidates all qualify: any of them
-  k_out = k_rem - __shfl_sync(kFull, gt, src);
+  const uint32_t gt_src = __shfl_sync(kFull, gt, src);
+  k_out = k_rem - gt_src;
+  n_equal = __shfl_sync(kFull, ge, src) - gt_src;
   return __shfl_sync(kFull, v, src);
 }
 
@@ -162,41 +164,59 @@ __device__ __forceinline__ void mark_top_keys(const unsigned long long* keys, in
   int rem = range ? 64 - __clzll((long long)range) : 0;
   unsigned long long top = 0;
   uint32_t k_rem = (uint32_t)k;
+  uint32_t n_equal = (uint32_t)n;                      // keys equal to the k-th largest (all of them when range == 0)
+  bool first = true;
   while (rem > 0) {
     const int w = rem < kDigitBits ? rem : kDigitBits, shift = rem - w, n_bins = 1 << w;
     for (int i = tid; i < n_bins; i += kThreads) sc.hist[i] = 0;
     if (tid == 0) sc.small_n = 0;
     __syncthreads();
-    for (int i = tid; i < n; i += kThreads) {
-      const unsigned long long x = keys[i] - base;
-      if (((x >> 1) >> (rem - 1)) == top) atomicAdd(&sc.hist[(uint32_t)(x >> shift) & (uint32_t)(n_bins - 1)], 1u);
+    if (first) {                                       // every key counts and has no bits above the digit
+      for (int i = tid; i < n; i += kThreads) atomicAdd(&sc.hist[(uint32_t)((keys[i] - base) >> shift)], 1u);
+    } else {
+      for (int i = tid; i < n; i += kThreads) {
+        const unsigned long long x = keys[i] - base;
+        if (((x >> 1) >> (rem - 1)) == top) atomicAdd(&sc.hist[(uint32_t)(x >> shift) & (uint32_t)(n_bins - 1)], 1u);
+      }
     }
+    first = false;
     __syncthreads();
     find_digit_desc<kThreads>(sc.hist, n_bins, k_rem, sc.warp_tot, sc.sel);
     top = (top << w) | sc.sel[0];
     k_rem = sc.sel[1];
     const uint32_t live = sc.sel[2];
+    n_equal = live;                                    // exact once no bits are left
     rem = shift;
     if (rem > 0 && live <= (uint32_t)kSmallList) {     // few candidates: one warp ranks their remaining bits
       for (int i = tid; i < n; i += kThreads) {
         const unsigned long long x = keys[i] - base;
-        if (((x >> 1) >> (rem - 1)) == top) sc.small[atomicAdd(&sc.small_n, 1u)] = x;
+        if ((x >> rem) == top) sc.small[atomicAdd(&sc.small_n, 1u)] = x;
       }
       __syncthreads();
       if (warp == 0) {
-        uint32_t k_out;
-        const unsigned long long v = warp_rank_select(lane < (int)live ? sc.small[lane] : 0ull, (int)live, k_rem, lane, k_out);
-        if (lane == 0) { sc.sel_x = v; sc.sel[1] = k_out; }
+        uint32_t k_out, n_eq_out;
+        const unsigned long long v = warp_rank_select(lane < (int)live ? sc.small[lane] : 0ull, (int)live, k_rem, lane, k_out, n_eq_out);
+        if (lane == 0) { sc.sel_x = v; sc.sel[1] = k_out; sc.sel[2] = n_eq_out; }
       }
       __syncthreads();
       top = sc.sel_x;
       k_rem = sc.sel[1];
+      n_equal = sc.sel[2];
       rem = 0;
     }
     __syncthreads();                                   // sc.sel and sc.hist are rewritten by the next step
   }
-  // kth = the k-th largest key; k_rem = how many keys equal to it are admitted
+  // kth = the k-th largest key; k_rem of the n_equal keys equal to it are admitted, in ascending index order
   const unsigned long long kth = base + top;
+  if (k_rem == n_equal) {                              // no tie is cut (the usual case): everything >= kth is in
+    for (int base_i = r_lo; base_i < r_hi; base_i += 32) {
+      const int i = base_i + lane;
+      const unsigned imp_b = __ballot_sync(kFull, i < r_hi && keys[i] >= kth);
+      if (lane == 0) imp_mask[base_i >> 5] = imp_b;
+    }
+    __syncthreads();
+    return;
+  }
   int n_eq = 0;
   for (int i = r_lo + lane; i < r_hi; i += 32) n_eq += (keys[i] == kth);
 #pragma unroll
