@@ -147,7 +147,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
     uint32_t* arena = dyn_smem + 2 * a.mask_words;
     if (a.stage_sorted) { sorted = reinterpret_cast<int32_t*>(arena); arena += a.stage_words; }
     if (a.stage_sig) {
-      for (int i = tid; i < L * W; i += kThreads) arena[i] = __ldg(sig + i);
+      _Pragma("unroll 8") for (int i = tid; i < L * W; i += kThreads) arena[i] = __ldg(sig + i);
       sig = arena;
       arena += a.stage_words * W;
     }
@@ -155,10 +155,10 @@ select_segment_kernel(Shape s, SelectArgs a) {
       unsigned long long* ks = reinterpret_cast<unsigned long long*>(arena);
       sort_code = reinterpret_cast<uint32_t*>(arena);      // the keys are dead once the important set is marked
       if (a.keys) {
-        for (int i = tid; i < L; i += kThreads) ks[i] = keys[i];
+        _Pragma("unroll 8") for (int i = tid; i < L; i += kThreads) ks[i] = keys[i];
       } else {
         const double* imp = a.imp + (size_t)layer * s.T + t0;
-        for (int i = tid; i < L; i += kThreads) ks[i] = importance_key(imp[i], i, L, a.keep_initial, a.keep_recent);
+        _Pragma("unroll 8") for (int i = tid; i < L; i += kThreads) ks[i] = importance_key(__ldg(imp + i), i, L, a.keep_initial, a.keep_recent);
       }
       keys = ks;
     }
