@@ -83,6 +83,17 @@ importance_keys_kernel(Shape s, const double* __restrict__ imp, int keep_initial
   keys[gid] = importance_key(imp[gid], tok - t0, __ldg(s.cu_seqlens + seq + 1) - t0, keep_initial, keep_recent);
 }
 
+// sum over the GW lanes of this lane's group of popc(mine & theirs); lanes without a member hold zeros
+template <int W, int GW>
+__device__ __forceinline__ int group_and_popc(const uint32_t (&mine)[4]) {
+  int shared = 0;
+#pragma unroll
+  for (int u = 0; u < GW; ++u)
+#pragma unroll
+    for (int w = 0; w < W; ++w) shared += __popc(mine[w] & __shfl_sync(kFull, mine[w], u, GW));
+  return shared;
+}
+
 struct SelectArgs {
   const unsigned long long* keys;     // [n_layers][T] importance keys; or, when NULL,
   const double* imp;                  // [n_layers][T] importance values, turned into keys while they are staged
@@ -283,7 +294,7 @@ select_segment_kernel(Shape s, SelectArgs a) {
     if (m_max <= 16) {
       // Small buckets (the usual case: N/R is the compression ratio): 32 / gw buckets share a warp, gw = the power
       // of two that holds a bucket, one lane per member.  sum_{h set in t} n_h = sum over members u of
-      // popc(sig_t & sig_u), so cost(t) = m * popc(sig_t) - 2 * sum_u popc(sig_t & sig_u): m_max shuffles inside
+      // popc(sig_t & sig_u), so cost(t) = m * popc(sig_t) - 2 * sum_u popc(sig_t & sig_u): gw shuffles inside
       // the lane group.  |cost| <= 16 * 128 and t < 2^18, so (cost, t) packs into 31 bits and one warp-level
       // minimum per lane group picks the representative, ties to the lower token.
       int gw = 2;
@@ -308,10 +319,11 @@ select_segment_kernel(Shape s, SelectArgs a) {
         const int t = member ? sorted[lo + j] : 0;
         uint32_t mine[4] = {0u, 0u, 0u, 0u};
         _Pragma("unroll") for (int w = 0; w < W; ++w) mine[w] = member ? sig[(size_t)t * W + w] & head_mask(s.Hq, w) : 0u;
-        int ones = 0, shared = 0;
+        int ones = 0;
         _Pragma("unroll") for (int w = 0; w < W; ++w) ones += __popc(mine[w]);
-        for (int u = 0; u < m_max; ++u)            // lanes past a bucket's last member hold zeros and add nothing
-          _Pragma("unroll") for (int w = 0; w < W; ++w) shared += __popc(mine[w] & __shfl_sync(kFull, mine[w], u, gw));
+        // lanes past a bucket's last member hold zeros and add nothing
+        const int shared = gw == 8 ? group_and_popc<W, 8>(mine) : gw == 4 ? group_and_popc<W, 4>(mine)
+                         : gw == 16 ? group_and_popc<W, 16>(mine) : group_and_popc<W, 2>(mine);
         const int cost = m * ones - 2 * shared;
         const uint32_t key = member ? ((uint32_t)(cost + 4096) << 18) | (uint32_t)t : 0xFFFFFFFFu;
         const uint32_t best = __reduce_min_sync(gmask, key);
