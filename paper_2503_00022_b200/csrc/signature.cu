@@ -19,11 +19,6 @@ namespace kvc {
 namespace {
 
 constexpr int kSelectThreads = 512;
-#ifndef KVC_THETA_T8K
-#define KVC_THETA_T8K 256                      // threads of theta_select_kernel for rows of 4097..8192 tokens (measured:
-                                               // 256 threads x 32 keys 18.4 us, 512 x 16 20.3 us, 1024 x 8 21.6 us, 128 x 64 23.7 us
-                                               // for 1024 rows of 8192)
-#endif
 constexpr int kThetaBits = 12;                 // radix digit of theta_select_kernel
 constexpr int kThetaBins = 1 << kThetaBits;
 
@@ -36,9 +31,13 @@ __device__ __forceinline__ float key_to_float(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
-// kT threads, each holding up to kItems keys of the row: rows of up to kT * kItems tokens.
-template <int kT, int kItems>
-__global__ void __launch_bounds__(kT)
+// kT threads, each holding up to kItems keys of the row: rows of up to kT * kItems tokens.  kMinB: resident blocks per
+// SM the kernel is compiled for.  The kernel is a chain of short dependent steps, so what counts is how many rows an
+// SM works on at once and how many threads share a row: measured for 1024 rows of 8192 scores, 512 threads x 16 keys
+// at 4 blocks per SM (32 registers, a few spilled words) 16.2 us, 256 x 32 at 4 per SM 17.9 us, 512 x 16 at 2 per SM
+// 20.3 us, 1024 x 8 at 2 per SM 19.7 us, 128 x 64 23.7 us.
+template <int kT, int kItems, int kMinB>
+__global__ void __launch_bounds__(kT, kMinB)
 theta_select_kernel(Shape s, const float* __restrict__ scores, const int32_t* __restrict__ sig_keep,
                     float* __restrict__ theta) {
   __shared__ alignas(16) uint32_t hist[kThetaBins];
@@ -223,9 +222,12 @@ theta_stream_kernel(Shape s, const float* __restrict__ scores, const int32_t* __
 // The thresholds of the block's sequence sit in shared memory when all its tokens belong to one sequence (always,
 // with one sequence per batch); else every thread reads its own sequence's row.
 constexpr int kPackTok = 128;
+#ifndef KVC_PACK_MINB
+#define KVC_PACK_MINB 8                 // resident blocks per SM the pack kernel is compiled for (registers per thread)
+#endif
 
 template <bool kImportance>
-__global__ void __launch_bounds__(kPackTok)
+__global__ void __launch_bounds__(kPackTok, KVC_PACK_MINB)
 signature_pack_kernel(Shape s, const float* __restrict__ scores, const float* __restrict__ theta,
                       uint32_t* __restrict__ sigs, double* __restrict__ importance, int vec_ok) {
   extern __shared__ float4 tile4[];                   // [Hq][kPackTok] float
@@ -275,10 +277,10 @@ signature_pack_kernel(Shape s, const float* __restrict__ scores, const float* __
   if constexpr (kImportance) importance[(size_t)layer * s.T + tok] = __dadd_rn(total, 0.0);       // -0.0 -> +0.0
 }
 
-template <int kT, int kItems>
+template <int kT, int kItems, int kMinB>
 void launch_theta(const Shape& s, const float* scores, const int32_t* sig_keep, float* theta, unsigned blocks,
                   cudaStream_t stream) {
-  theta_select_kernel<kT, kItems><<<blocks, kT, 0, stream>>>(s, scores, sig_keep, theta);
+  theta_select_kernel<kT, kItems, kMinB><<<blocks, kT, 0, stream>>>(s, scores, sig_keep, theta);
 }
 
 }  // namespace
@@ -290,11 +292,11 @@ int launch_signature(const Shape& s, const float* scores, const int32_t* sig_kee
   if (!theta_in) {
     const unsigned blocks = (unsigned)s.n_layers * s.n_seqs * s.Hq;
     const int m = s.max_seqlen;
-    if (m <= 2048) launch_theta<256, 8>(s, scores, sig_keep, theta, blocks, stream);
-    else if (m <= 4096) launch_theta<256, 16>(s, scores, sig_keep, theta, blocks, stream);
-    else if (m <= 8192) launch_theta<KVC_THETA_T8K, 8192 / KVC_THETA_T8K>(s, scores, sig_keep, theta, blocks, stream);
-    else if (m <= 16384) launch_theta<512, 32>(s, scores, sig_keep, theta, blocks, stream);
-    else if (m <= 32768) launch_theta<1024, 32>(s, scores, sig_keep, theta, blocks, stream);
+    if (m <= 2048) launch_theta<256, 8, 8>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 4096) launch_theta<512, 8, 4>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 8192) launch_theta<512, 16, 4>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 16384) launch_theta<512, 32, 1>(s, scores, sig_keep, theta, blocks, stream);
+    else if (m <= 32768) launch_theta<1024, 32, 1>(s, scores, sig_keep, theta, blocks, stream);
     else {
       const size_t row_bytes = (size_t)m * sizeof(uint32_t);
       const int stage_row = row_bytes <= 200 * 1024;
