@@ -634,6 +634,13 @@ def run_ours(args, w):
             ghz = sus["clocks"]["sm_mhz"] * 1e-3
             roofline["sm_ghz_sustained"] = ghz
             roofline["launch_ms_x_ghz"] = launch_ms * ghz          # clock-independent cost of one sweep: Mcycles
+            # context: the other unit the sweeps load - one exponential per causal logit per sweep, 16 per clock per SM
+            # on the special-function unit at the sampled clock (a quarter of them are evaluated on the FMA pipe instead)
+            n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+            sfu_peak = n_sm * 16 * ghz * 1e9
+            roofline["exp_unit"] = {"exps_per_s": roofline["exps_per_s"], "sfu_peak_per_s": sfu_peak,
+                                    "frac_if_all_on_sfu": roofline["exps_per_s"] / sfu_peak,
+                                    "sfu_share_of_exps": 0.75}
     else:
         # fp32 FMA on the CUDA cores: 128 lanes x 2 flop per SM per clock at the SM clock sampled during the timed steps
         n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
